@@ -1,0 +1,266 @@
+"""ctypes binding of the IntSGD CPU oracle -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+
+The arithmetic lives in ``intsgd_oracle.cpp`` (plain single-threaded C++, fp32 operations
+rounded one by one, own Philox4x32-10).  This module compiles it with g++ on first use, exposes
+its functions and strings them together in the order of Algorithm 1 of the IntSGD paper
+(``OracleIntSGD``).  Only tests, the smoke check and the benchmark's CPU-baseline leg import it;
+it imports nothing from the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "intsgd_oracle.cpp"
+_LIB = _HERE / "liboracle_intsgd.so"
+
+GRAD_F32, GRAD_BF16 = 0, 1
+PAYLOAD_I32, PAYLOAD_I8 = 0, 1
+ROUND_RANDOM, ROUND_NEAREST = 0, 1
+INT32_MAX = 2**31 - 1
+
+
+def build(force: bool = False) -> Path:
+    """Compile the oracle (g++, no FMA contraction, no fast-math)."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".{os.getpid()}.tmp")
+        subprocess.run(
+            ["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-Wall",
+             "-shared", "-fPIC", "-o", str(tmp), str(_SRC)], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(str(build()))
+        L = _lib
+        u32p, f32p, i32p = C.POINTER(C.c_uint32), C.POINTER(C.c_float), C.POINTER(C.c_int32)
+        f64p, u64p = C.POINTER(C.c_double), C.POINTER(C.c_uint64)
+        L.orc_philox4x32_10.argtypes = [u32p, u32p, u32p]
+        L.orc_philox4x32_10.restype = None
+        L.orc_draw_word.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64]
+        L.orc_draw_word.restype = C.c_uint32
+        L.orc_uniform_from_word.argtypes = [C.c_uint32]
+        L.orc_uniform_from_word.restype = C.c_float
+        L.orc_int_round.argtypes = [C.c_float, C.c_float]
+        L.orc_int_round.restype = C.c_int32
+        L.orc_int_round_nearest.argtypes = [C.c_float]
+        L.orc_int_round_nearest.restype = C.c_int32
+        L.orc_limit_as_float.argtypes = [C.c_int64]
+        L.orc_limit_as_float.restype = C.c_float
+        L.orc_scale.argtypes = [C.c_int64, C.c_int32, C.c_double, C.c_double, C.c_double,
+                                C.c_double, C.c_double, f64p, f64p, f32p, f32p]
+        L.orc_scale.restype = None
+        L.orc_scale_block.argtypes = [C.c_int64, C.c_int64, C.c_int32, C.c_double, C.c_double,
+                                      C.c_double, C.c_double, C.c_double, f64p, f64p, f32p, f32p]
+        L.orc_scale_block.restype = None
+        L.orc_encode.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_float, C.c_int64,
+                                 C.c_int, C.c_int, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
+                                 C.c_void_p, u64p, u64p]
+        L.orc_encode.restype = None
+        L.orc_aggregate.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64,
+                                    C.c_float, C.c_void_p, C.c_void_p, f64p, u64p, i32p]
+        L.orc_aggregate.restype = None
+        L.orc_exact_step.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64,
+                                     C.c_double, C.c_void_p, f64p]
+        L.orc_exact_step.restype = None
+        L.orc_sqdiff.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
+        L.orc_sqdiff.restype = C.c_double
+        L.orc_step_window.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64,
+                                      C.c_int64, C.c_float, C.c_float, C.c_int64, C.c_int, C.c_int,
+                                      C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      f64p, u64p, u64p, u64p, i32p]
+        L.orc_step_window.restype = None
+    return _lib
+
+
+# --------------------------------------------------------------------------- small helpers
+def _ptr(a: np.ndarray | None) -> C.c_void_p:
+    return C.c_void_p(None) if a is None else C.c_void_p(a.ctypes.data)
+
+
+def _grad_dtype(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return GRAD_F32
+    if a.dtype == np.uint16:  # bf16 bit patterns
+        return GRAD_BF16
+    raise TypeError(f"gradient must be float32 or uint16 (bf16 bits), got {a.dtype}")
+
+
+def _ptr_array(arrs) -> C.Array:
+    return (C.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+
+
+def default_clip_limit(n: int, payload_dtype: int) -> int:
+    """int8 wire: 127.  int32 wire: floor((2^31 - 1) / n), so the sum of n payloads fits."""
+    return 127 if payload_dtype == PAYLOAD_I8 else INT32_MAX // n
+
+
+def philox4x32_10(ctr, key) -> tuple[int, int, int, int]:
+    c = (C.c_uint32 * 4)(*ctr)
+    k = (C.c_uint32 * 2)(*key)
+    o = (C.c_uint32 * 4)()
+    lib().orc_philox4x32_10(c, k, o)
+    return tuple(int(v) for v in o)
+
+
+def draw_word(seed: int, step: int, worker: int, j: int) -> int:
+    return int(lib().orc_draw_word(seed, step, worker, j))
+
+
+def uniform_from_word(w: int) -> float:
+    return float(lib().orc_uniform_from_word(w))
+
+
+def int_round(y: float, u: float) -> int:
+    return int(lib().orc_int_round(y, u))
+
+
+def int_round_nearest(y: float) -> int:
+    return int(lib().orc_int_round_nearest(y))
+
+
+def limit_as_float(L: int) -> float:
+    return float(lib().orc_limit_as_float(L))
+
+
+def scale(d, n, eta, beta, eps, r_prev, dx2):
+    """(r_k, alpha_k in fp64, alpha_k rounded to fp32, c_k = eta/(n alpha_k) in fp32)."""
+    r, a64 = C.c_double(), C.c_double()
+    a32, c32 = C.c_float(), C.c_float()
+    lib().orc_scale(d, n, eta, beta, eps, r_prev, dx2, C.byref(r), C.byref(a64), C.byref(a32),
+                    C.byref(c32))
+    return r.value, a64.value, np.float32(a32.value), np.float32(c32.value)
+
+
+def scale_block(d, d_l, n, eta, beta, eps, r_prev, dx2):
+    r, a64 = C.c_double(), C.c_double()
+    a32, c32 = C.c_float(), C.c_float()
+    lib().orc_scale_block(d, d_l, n, eta, beta, eps, r_prev, dx2, C.byref(r), C.byref(a64),
+                          C.byref(a32), C.byref(c32))
+    return r.value, a64.value, np.float32(a32.value), np.float32(c32.value)
+
+
+def encode(grad, alpha, *, worker, step, seed, n=None, clip_limit=None,
+           payload_dtype=PAYLOAD_I32, rounding=ROUND_RANDOM, j0=0, u_inject=None):
+    """Int(alpha * grad) for one worker over coordinates [j0, j0 + len(grad)).
+
+    Returns (payload, clip_count, nonfinite_count)."""
+    grad = np.ascontiguousarray(grad)
+    if clip_limit is None:
+        clip_limit = default_clip_limit(n, payload_dtype)
+    out = np.empty(grad.shape[0], dtype=np.int8 if payload_dtype == PAYLOAD_I8 else np.int32)
+    clip, nonf = C.c_uint64(0), C.c_uint64(0)
+    if u_inject is not None:
+        u_inject = np.ascontiguousarray(u_inject, dtype=np.float32)
+    lib().orc_encode(_ptr(grad), _grad_dtype(grad), j0, grad.shape[0], float(alpha),
+                     int(clip_limit), payload_dtype, rounding, seed, step, worker,
+                     _ptr(u_inject), _ptr(out), C.byref(clip), C.byref(nonf))
+    return out, clip.value, nonf.value
+
+
+def aggregate(payloads, x, c, *, want_agg=True):
+    """Sum the payloads, decode with c = eta/(n alpha), update x in place.
+
+    Returns (agg or None, dx2, agg_overflow, max_abs_agg)."""
+    payloads = [np.ascontiguousarray(p) for p in payloads]
+    pd = PAYLOAD_I8 if payloads[0].dtype == np.int8 else PAYLOAD_I32
+    count = payloads[0].shape[0]
+    assert x.dtype == np.float32 and x.flags.c_contiguous
+    agg = np.empty(count, dtype=np.int32) if want_agg else None
+    dx2, ovf, mx = C.c_double(), C.c_uint64(0), C.c_int32(0)
+    lib().orc_aggregate(_ptr_array(payloads), pd, len(payloads), count, float(c), _ptr(x),
+                        _ptr(agg), C.byref(dx2), C.byref(ovf), C.byref(mx))
+    return agg, dx2.value, ovf.value, mx.value
+
+
+def exact_step(grads, x, eta):
+    """Init line of Algorithm 1: x <- x - eta * mean_i g_i.  Returns dx2."""
+    grads = [np.ascontiguousarray(g) for g in grads]
+    dx2 = C.c_double()
+    lib().orc_exact_step(_ptr_array(grads), _grad_dtype(grads[0]), len(grads), x.shape[0],
+                         float(eta), _ptr(x), C.byref(dx2))
+    return dx2.value
+
+
+def sqdiff(x, x_prev) -> float:
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    x_prev = np.ascontiguousarray(x_prev, dtype=np.float32)
+    return float(lib().orc_sqdiff(_ptr(x), _ptr(x_prev), x.shape[0]))
+
+
+def step_window(grads, x, alpha, c, *, step, seed, j0=0, clip_limit=None,
+                payload_dtype=PAYLOAD_I32, rounding=ROUND_RANDOM, want_agg=True):
+    """One compressed step on coordinates [j0, j0 + len(x)) with (alpha, c) given.
+
+    ``grads[i]`` and ``x`` hold only the window.  Updates x in place and returns a dict with
+    agg, dx2 (of the window), clip_count[n], nonfinite, agg_overflow, max_abs_agg."""
+    grads = [np.ascontiguousarray(g) for g in grads]
+    n, count = len(grads), x.shape[0]
+    if clip_limit is None:
+        clip_limit = default_clip_limit(n, payload_dtype)
+    agg = np.empty(count, dtype=np.int32) if want_agg else None
+    scratch = np.empty(n * count, dtype=np.int32)
+    clip = (C.c_uint64 * n)()
+    dx2, nonf, ovf, mx = C.c_double(), C.c_uint64(0), C.c_uint64(0), C.c_int32(0)
+    lib().orc_step_window(_ptr_array(grads), _grad_dtype(grads[0]), n, j0, count, float(alpha),
+                          float(c), int(clip_limit), payload_dtype, rounding, seed, step, _ptr(x),
+                          _ptr(agg), _ptr(scratch), C.byref(dx2), clip, C.byref(nonf),
+                          C.byref(ovf), C.byref(mx))
+    return dict(agg=agg, dx2=dx2.value, clip_count=[int(v) for v in clip], nonfinite=nonf.value,
+                agg_overflow=ovf.value, max_abs_agg=mx.value)
+
+
+class OracleIntSGD:
+    """Algorithm 1 as a state machine: (r, dx2, step) carried between calls.
+
+    ``step == 0`` is the exact first communication (Init line); every later step computes r_k and
+    alpha_k (Proposition 2), rounds, sums, decodes and updates.  ``alpha_c`` lets a caller impose
+    the fp32 (alpha, c) pair actually used for the vector part (lock-step comparison with an
+    implementation whose norm reduction has another summation order); the oracle's own r and
+    alpha are still computed and returned.
+    """
+
+    def __init__(self, n, d, *, beta=0.9, eps=1e-8, seed=0, payload_dtype=PAYLOAD_I32,
+                 clip_limit=None, rounding=ROUND_RANDOM):
+        self.n, self.d = n, d
+        self.beta, self.eps, self.seed = beta, eps, seed
+        self.payload_dtype, self.rounding = payload_dtype, rounding
+        self.clip_limit = default_clip_limit(n, payload_dtype) if not clip_limit else clip_limit
+        self.r = 0.0
+        self.dx2 = 0.0
+        self.step = 0
+
+    def exact_step(self, grads, x, eta):
+        dx2 = exact_step(grads, x, eta)
+        self.dx2 = dx2
+        self.step += 1
+        return dict(dx2=dx2)
+
+    def scale(self, eta, dx2=None):
+        """Advance r with the stored (or given) squared step length and return the scale."""
+        r, a64, a32, c32 = scale(self.d, self.n, eta, self.beta, self.eps, self.r,
+                                 self.dx2 if dx2 is None else dx2)
+        self.r = r
+        return r, a64, a32, c32
+
+    def int_step(self, grads, x, eta, *, alpha_c=None, dx2_in=None, want_agg=True):
+        r, a64, a32, c32 = self.scale(eta, dx2_in)
+        alpha, c = (a32, c32) if alpha_c is None else alpha_c
+        out = step_window(grads, x, alpha, c, step=self.step, seed=self.seed, j0=0,
+                          clip_limit=self.clip_limit, payload_dtype=self.payload_dtype,
+                          rounding=self.rounding, want_agg=want_agg)
+        self.dx2 = out["dx2"]
+        self.step += 1
+        out.update(r=r, alpha64=a64, alpha=a32, c=c32)
+        return out
