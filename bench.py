@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the fused IntSGD step (gradient elements/s and HBM roofline fraction).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one whole IntSGD iteration -- scale, encode, integer sum, decode, update, next-norm --
+over n workers' gradients of length d that are already in device memory (`value`), and the same
+step through the host-buffer entry point with the copies inside the timed region (`e2e`).
+Workload: the large-model bucket (d = 2^26 fp32 N(0, 1e-3^2), n = 16 workers, int32 aggregate,
+fused single-pass path).  With N > 1 (torchrun) every rank runs an independent replica on its own
+GPU: the path has no exchange step on one node, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "fused IntSGD step throughput"
+UNIT = "gradient elements/s"
+HBM_FALLBACK_GBS = 6650.0
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=50)
+    p.add_argument("--warmup", type=int, default=5)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--log2d", type=int, default=26)
+    p.add_argument("--workers", type=int, default=16)
+    p.add_argument("--payload", default="int32", choices=["int32", "int8"])
+    p.add_argument("--grad", default="f32", choices=["f32", "bf16"])
+    p.add_argument("--mode", default="fused", choices=["fused", "two_kernel"])
+    p.add_argument("--rounding", default="random", choices=["random", "nearest"])
+    p.add_argument("--eta", type=float, default=0.1)
+    p.add_argument("--e2e-steps", type=int, default=3)
+    p.add_argument("--cpu-sample-log2", type=int, default=24,
+                   help="coordinates of the oracle sample (all workers), as a power of two")
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-e2e", action="store_true")
+    p.add_argument("--threads", type=int, default=0)
+    p.add_argument("--blocks-per-sm", type=int, default=0)
+    return p.parse_args()
+
+
+# ------------------------------------------------------------------------------------------
+def measured_hbm_peak():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            return float(json.loads(f.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return HBM_FALLBACK_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for (t, line) in self.lines:
+            if t0 is not None and not (t0 <= t <= t1 + 0.15):
+                continue
+            parts = [s.strip() for s in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def algorithmic_bytes_per_coordinate(n, grad_bytes, payload_bytes, mode):
+    """Bytes that must cross HBM per coordinate: n gradient reads, x read + write, aggregate write
+    (fused); plus n payload writes and n payload reads on the two-kernel path."""
+    base = n * grad_bytes + 12
+    if mode == "two_kernel":
+        base += 2 * n * payload_bytes
+    return base
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_sample_throughput(n, d, sample_log2, grad_dtype, payload, rounding, seed=77):
+    """Time the CPU oracle, as it stands, on one step over the first 2^sample_log2 coordinates of
+    all n workers.  Returns (elements/s, seconds, description)."""
+    import numpy as np
+    import oracle
+    from paper_2102_08374_b200 import synth
+    w = min(d, 1 << sample_log2)
+    grads = [synth.bucket_gradient(i, w) for i in range(n)]
+    if grad_dtype == "bf16":
+        grads = [synth.to_bf16_bits(g) for g in grads]
+    x = synth.iterate(w)
+    pd = oracle.PAYLOAD_I8 if payload == "int8" else oracle.PAYLOAD_I32
+    rd = oracle.ROUND_NEAREST if rounding == "nearest" else oracle.ROUND_RANDOM
+    oracle.step_window([g[:1024] for g in grads], x[:1024].copy(), np.float32(700.0), np.float32(1e-5), step=1,
+                       seed=seed, payload_dtype=pd, rounding=rd)     # load the library, touch the code
+    t = time.perf_counter()
+    oracle.step_window(grads, x, np.float32(700.0), np.float32(1e-5), step=1, seed=seed, payload_dtype=pd, rounding=rd)
+    dt = time.perf_counter() - t
+    return n * w / dt, dt, f"one step on the first 2^{sample_log2} coordinates of all {n} workers ({n * w} elements)"
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, single-threaded, on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n, d = args.workers, 1 << args.log2d
+    sample_log2 = min(args.cpu_sample_log2, 22)
+    for _ in range(max(args.warmup, 0) and 1):
+        oracle_sample_throughput(n, d, 16, args.grad, args.payload, args.rounding)
+    times, elems = [], 0
+    for _ in range(max(1, min(args.steps, 8))):
+        v, dt, desc = oracle_sample_throughput(n, d, sample_log2, args.grad, args.payload, args.rounding)
+        times.append(dt)
+        elems = n * min(d, 1 << sample_log2)
+    value = elems * len(times) / sum(times)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": len(times), "warmup": 1, "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(args):
+    return {"workload": f"large-model bucket: d=2^{args.log2d} {args.grad} N(0,1e-3^2), n={args.workers} workers, "
+                        f"{args.payload} wire, {args.mode} path, {args.rounding} rounding",
+            "d": 1 << args.log2d, "n_workers": args.workers, "grad_dtype": args.grad, "payload": args.payload,
+            "mode": args.mode, "rounding": args.rounding,
+            "l2": "inputs larger than L2 (gradients alone are n*d*4 bytes); no flush between iterations"}
+
+
+# ------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2102_08374_b200 as pkg
+    from paper_2102_08374_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    n, d = args.workers, 1 << args.log2d
+    grad_dtype = pkg.GRAD_BF16 if args.grad == "bf16" else pkg.GRAD_F32
+    payload_dtype = pkg.PAYLOAD_I8 if args.payload == "int8" else pkg.PAYLOAD_I32
+    rounding = pkg.ROUND_NEAREST if args.rounding == "nearest" else pkg.ROUND_RANDOM
+    mode = pkg.MODE_TWO_KERNEL if args.mode == "two_kernel" else pkg.MODE_FUSED
+    gb, pb = (2 if args.grad == "bf16" else 4), (1 if args.payload == "int8" else 4)
+
+    grads = synth.bucket_gradients_device(n, d, device, seed_base=500 + 1000 * rank,
+                                          dtype=torch.bfloat16 if args.grad == "bf16" else None)
+    x = synth.iterate_device(d, device)
+    agg = torch.empty(d, dtype=torch.int32, device=device)
+    scratch = None
+    if mode == pkg.MODE_TWO_KERNEL:
+        scratch = [torch.empty(d, dtype=torch.int8 if pb == 1 else torch.int32, device=device) for _ in range(n)]
+    lib = pkg.IntSGD(n, d, grad_dtype=grad_dtype, payload_dtype=payload_dtype, rounding=rounding, seed=2102_08374,
+                     device=local_rank)
+    lib.intsgd_set_launch(args.threads, args.blocks_per_sm)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def step(k):
+        lib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=pkg.MODE_EXACT if k == 0 else mode,
+                        payload_scratch=scratch, stream=stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # step 0 is the exact first communication; then W warm-up steps; then K timed steps
+    step(0)
+    for k in range(1, 1 + max(args.warmup, 3)):
+        step(k)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    K = args.steps
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    launches0 = lib.intsgd_launch_count()
+    barrier()
+    t_wall0 = time.time()
+    events[0].record()
+    for k in range(K):
+        step(1000 + k)
+        events[k + 1].record()
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    launches = lib.intsgd_launch_count() - launches0
+    barrier()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    total_ms = events[0].elapsed_time(events[K])
+    per_step_ms = [events[k].elapsed_time(events[k + 1]) for k in range(K)]
+    st = lib.intsgd_get_stats()
+    if dist is not None:
+        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    value = world * n * d * K / (total_ms * 1e-3)
+    bytes_per_launch = algorithmic_bytes_per_coordinate(n, gb, pb, args.mode) * d
+    avg_ms = statistics.mean(per_step_ms)
+    peak, peak_kind = measured_hbm_peak()
+    achieved = bytes_per_launch / (avg_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_source": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
+                "algorithmic_bytes_per_launch": bytes_per_launch, "kernel_ms_avg": avg_ms,
+                "kernel_ms_median": statistics.median(per_step_ms),
+                "note": "per-step CUDA-event time (one-thread scale kernel + the vector kernel(s))"}
+
+    # ---- end to end through the host-buffer entry point (rank-local; max over ranks) ----
+    e2e = None
+    if not args.no_e2e and mode == pkg.MODE_FUSED:
+        hg = [torch.empty(d, dtype=g.dtype, pin_memory=True) for g in grads]
+        for h, g in zip(hg, grads):
+            h.copy_(g)
+        hx = torch.empty(d, dtype=torch.float32, pin_memory=True)
+        hx.copy_(x)
+        hagg = torch.empty(d, dtype=torch.int32, pin_memory=True)
+        lib.intsgd_step_host(hg, hx, hagg, eta_k=args.eta, mode=mode, stream=stream)      # allocates staging
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record()
+        for _ in range(args.e2e_steps):
+            lib.intsgd_step_host(hg, hx, hagg, eta_k=args.eta, mode=mode, stream=stream)
+        ev1.record()
+        torch.cuda.synchronize()
+        e2e_ms = ev0.elapsed_time(ev1)
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": world * n * d * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": n * d * gb + d * 4, "d2h_bytes_per_step": d * 8,
+               "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,
+               "call": "intsgd_step_host (pinned host gradients, x and aggregate; copies inside the timed region)"}
+        del hg, hx, hagg
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, dt, desc = oracle_sample_throughput(n, d, args.cpu_sample_log2, args.grad, args.payload, args.rounding)
+        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": dt}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+            "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if args.grad == "f32" else "bf16->f32", "data": "synthetic", "config": workload_config(args),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+            "hbm_gbs_algorithmic": achieved * world,
+            "state": {"alpha": st["alpha"], "r": st["r"], "max_abs_agg": st["max_abs_agg"],
+                      "clipped": sum(st["clip_count"]), "step": st["step"]},
+        }
+        print(json.dumps(line))
+    lib.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,175 @@
+/*
+ * intsgd.h -- C ABI of the IntSGD step library for NVIDIA B200 (sm_100a).
+ *
+ * One IntSGD iteration (Mishchenko, Wang, Kovalev, Richtarik, "IntSGD: Adaptive Floatless
+ * Compression of Stochastic Gradients", Algorithm 1) for n simulated workers whose gradient
+ * vectors of length d sit in the memory of ONE GPU:
+ *
+ *     r_k     = beta r_{k-1} + (1 - beta) ||x^k - x^{k-1}||^2          (Algorithm 1, moving average)
+ *     alpha_k = sqrt(d) / sqrt(2 n r_k / eta_k^2 + eps^2)              (Proposition 2)
+ *     q_i     = Int(alpha_k g_i)   Int(t) = floor(t) + Bernoulli(t - floor(t))   (Section 2)
+ *     S       = sum_i q_i          exact integer sum                   (Algorithm 1, aggregate)
+ *     x^{k+1} = x^k - eta_k S / (n alpha_k)                            (Algorithm 1, estimator + update)
+ *
+ * Conventions
+ *  - Every vector pointer is a DEVICE pointer owned by the caller unless the name says "host".
+ *    The library never frees or keeps them.  Pointers must be aligned to their element size;
+ *    16-byte aligned pointers take the vector path, others a slower element-wise path.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All vector work is
+ *    enqueued on it and returns without synchronising; only create / destroy / get_stats /
+ *    get_state / set_state / step_host synchronise.
+ *  - Every call returns an int status: 0 = INTSGD_OK, negative = error.  Nothing throws or
+ *    aborts.  intsgd_last_error() gives a message for the last failing call on that context.
+ *  - Clipping and integer overflow are not errors: they are counted (intsgd_stats).
+ *  - A context is not thread-safe; distinct contexts are independent.  Calls on one context
+ *    must be issued on one stream (or be ordered by the caller).
+ *  - The random stream is counter-based: Philox4x32-10 (Salmon et al., SC'11) with
+ *    key = (seed low, seed high), counter = (b low, b high, worker, step), b = j / 4, and
+ *    coordinate j uses output word j mod 4.  u = (word >> 8) * 2^-24; Int rounds up iff
+ *    u < fl32(y - floor(y)) with y = fl32(alpha * g).  Results do not depend on the launch shape.
+ *  - fp32 arithmetic of the vector part is unfused (separately rounded multiply and subtract).
+ */
+#ifndef INTSGD_H_
+#define INTSGD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define INTSGD_MAX_WORKERS 64
+
+/* status codes */
+#define INTSGD_OK                    0
+#define INTSGD_ERR_INVALID_ARG      -1   /* null pointer, n or d out of range, eta <= 0, bad enum */
+#define INTSGD_ERR_ALIGN            -2   /* pointer not aligned to its element size */
+#define INTSGD_ERR_CUDA             -3   /* a CUDA runtime call failed; see intsgd_last_error */
+#define INTSGD_ERR_SCALE_NONFINITE  -4   /* alpha_k or c_k not finite or not positive; step not applied */
+#define INTSGD_ERR_UNSUPPORTED      -5   /* valid request this build does not implement */
+
+/* enums (plain ints in the structs) */
+#define INTSGD_GRAD_F32      0
+#define INTSGD_GRAD_BF16     1
+#define INTSGD_PAYLOAD_I32   0
+#define INTSGD_PAYLOAD_I8    1
+#define INTSGD_ROUND_RANDOM  0   /* Int(t) of Section 2 */
+#define INTSGD_ROUND_NEAREST 1   /* "IntSGD (Determ.)" of Section 5.1: nearest, ties to even */
+#define INTSGD_MODE_EXACT      0 /* Algorithm 1, Init line: x <- x - eta (1/n) sum_i g_i, uncompressed */
+#define INTSGD_MODE_TWO_KERNEL 1 /* encode every worker to a payload buffer, then aggregate */
+#define INTSGD_MODE_FUSED      2 /* one pass, payloads never reach memory */
+
+typedef struct intsgd_ctx intsgd_ctx;   /* opaque; owns only a small device state block and
+                                           a few KiB of reduction scratch */
+
+typedef struct intsgd_config {
+    int32_t  n;              /* workers, 1 .. INTSGD_MAX_WORKERS */
+    int32_t  grad_dtype;     /* INTSGD_GRAD_* */
+    int64_t  d;              /* coordinates, 1 .. 2^40 */
+    int32_t  payload_dtype;  /* INTSGD_PAYLOAD_*: the wire type; the aggregate is always int32 */
+    int32_t  rounding;       /* INTSGD_ROUND_* */
+    double   beta;           /* moving-average factor in [0, 1); paper default 0.9 */
+    double   eps;            /* safeguard >= 0 (enters as eps^2); paper default 1e-8 */
+    uint64_t seed;           /* Philox key */
+    int64_t  clip_limit;     /* symmetric limit L on each payload value; 0 = default:
+                                int8 wire -> 127; int32 wire -> floor((2^31 - 1) / n), so that the
+                                aggregate of n payloads fits the wire type (Section 5.1).
+                                Must satisfy n * L <= 2^31 - 1. */
+    int32_t  device;         /* CUDA device ordinal */
+    int32_t  reserved;       /* must be 0 */
+} intsgd_config;
+
+/* The resumable scalar state.  With x it is everything needed to continue bit-exactly. */
+typedef struct intsgd_state {
+    double   r;       /* moving average r_k after the last intsgd_scale */
+    double   dx2;     /* ||x^{k+1} - x^k||^2 left by the last step (or intsgd_sqdiff) */
+    float    alpha;   /* alpha_k used by the last / next encode */
+    float    c;       /* eta_k / (n alpha_k), the decode factor */
+    uint32_t step;    /* 0-based index of the NEXT step (the Philox counter word) */
+    int32_t  status;  /* INTSGD_OK or INTSGD_ERR_SCALE_NONFINITE from the last intsgd_scale */
+} intsgd_state;
+
+/* Counters describe the work enqueued since the last intsgd_scale (one step). */
+typedef struct intsgd_stats {
+    intsgd_state state;
+    uint64_t clip_count[INTSGD_MAX_WORKERS]; /* per worker: coordinates with !(|alpha g| <= L) */
+    uint64_t nonfinite;      /* coordinates (all workers) whose alpha * g is NaN or +-Inf */
+    uint64_t agg_overflow;   /* int8 wire only: coordinates whose sum is outside [-127, 127] */
+    int32_t  max_abs_agg;    /* max_j |S_j| ("max integer in the aggregated vector", Appendix C.5) */
+    int32_t  reserved;
+} intsgd_stats;
+
+/* Lifetime.  create selects cfg->device, allocates the state block (r = 0, dx2 = 0, step = 0)
+ * and validates cfg.  destroy frees it; the caller must have synchronised its streams. */
+int intsgd_create(intsgd_ctx** out, const intsgd_config* cfg);
+int intsgd_destroy(intsgd_ctx* ctx);
+
+/* Algorithm 1, moving-average and scale lines (Proposition 2).  Enqueues a one-thread kernel:
+ * r <- beta r + (1 - beta) dx2;  alpha <- fp32(sqrt(d) / sqrt(2 n r / eta^2 + eps^2));
+ * c <- fp32(eta / (n alpha)), all in fp64 with separately rounded operations.
+ * dx2_override < 0: use the dx2 left in the state by the previous step; >= 0: use this value.
+ * Also clears the per-step counters.  eta_k must be finite and > 0 (else INVALID_ARG).
+ * If alpha or c is not finite and positive (r = 0 with eps = 0), the state keeps its old r, status
+ * becomes INTSGD_ERR_SCALE_NONFINITE, and the vector kernels of this step do nothing; the
+ * condition is reported by intsgd_get_stats / intsgd_get_state (this call is asynchronous). */
+int intsgd_scale(intsgd_ctx* ctx, double eta_k, double dx2_override, void* stream);
+
+/* Helper for a caller that holds two iterates: state.dx2 <- ||x - x_prev||^2
+ * (fp32 differences, fp64 sum; Algorithm 1, argument of the moving average). */
+int intsgd_sqdiff(intsgd_ctx* ctx, const float* x, const float* x_prev, void* stream);
+
+/* Algorithm 1, "scale and round the local gradient", for one worker:
+ * payload[j] = clip(Int(alpha g[j])), j in [0, d).  grad: d values of cfg.grad_dtype;
+ * payload: d values of cfg.payload_dtype.  alpha_override = NaN: use the state's alpha;
+ * otherwise use this value.  Adds to clip_count[worker] and nonfinite. */
+int intsgd_encode(intsgd_ctx* ctx, int32_t worker, const void* grad, void* payload,
+                  float alpha_override, void* stream);
+
+/* Algorithm 1, aggregate + estimator + update in one pass over memory:
+ * S_j = sum_i payloads[i][j];  x_j <- x_j - c S_j;  agg[j] = S_j (agg may be NULL);
+ * state.dx2 <- ||x_new - x_old||^2;  state.step += 1.
+ * payloads: HOST array of n device pointers (read during the call only). */
+int intsgd_aggregate(intsgd_ctx* ctx, const void* const* payloads, float* x, int32_t* agg,
+                     void* stream);
+
+/* One whole step k: scale (unless mode is EXACT), then
+ *   EXACT      : x <- x - eta (1/n) sum_i g_i in fp32, workers added in order 0..n-1
+ *                (Algorithm 1, Init line); r is left unchanged; no payloads, no counters.
+ *   TWO_KERNEL : encode all workers into payload_scratch[i] (n device buffers of d payload
+ *                values, caller-owned), then aggregate.
+ *   FUSED      : encode, sum, decode and update in one kernel; payload_scratch ignored.
+ * grads, payload_scratch: HOST arrays of n device pointers.  agg may be NULL.
+ * Leaves state.dx2 = ||x^{k+1} - x^k||^2 and advances state.step. */
+int intsgd_step(intsgd_ctx* ctx, const void* const* grads, void* const* payload_scratch,
+                float* x, int32_t* agg, double eta_k, int32_t mode, void* stream);
+
+/* The same step for a caller whose buffers are in HOST memory (pinned memory recommended):
+ * copies the n gradients and x to device staging buffers owned by the context (allocated on
+ * first use: n*d gradient values + d floats + d int32), runs intsgd_step, copies x (and agg if
+ * not NULL) back, and synchronises the stream before returning. */
+int intsgd_step_host(intsgd_ctx* ctx, const void* const* host_grads, float* host_x,
+                     int32_t* host_agg, double eta_k, int32_t mode, void* stream);
+
+/* Synchronise the context's last stream and read the state and counters.  Returns
+ * INTSGD_ERR_SCALE_NONFINITE if the last intsgd_scale failed that way (out is still filled). */
+int intsgd_get_stats(intsgd_ctx* ctx, intsgd_stats* out);
+int intsgd_get_state(intsgd_ctx* ctx, intsgd_state* out);
+/* Overwrite the scalar state (checkpoint resume; tests that impose alpha and c). */
+int intsgd_set_state(intsgd_ctx* ctx, const intsgd_state* in);
+
+/* Tuning knob: threads per block (multiple of 32, <= 1024) and resident blocks per SM used to
+ * size the grids of the vector kernels.  0 keeps the built-in value.  Results do not depend on
+ * it except the summation order of dx2. */
+int intsgd_set_launch(intsgd_ctx* ctx, int32_t threads_per_block, int32_t blocks_per_sm);
+
+/* Number of kernels this library has launched on the context since creation. */
+int64_t intsgd_launch_count(const intsgd_ctx* ctx);
+
+/* Static, NUL-terminated description of the last failing call ("" if none); never NULL.
+ * ctx may be NULL to read the message of a failed intsgd_create on this thread. */
+const char* intsgd_last_error(const intsgd_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* INTSGD_H_ */

@@ -1,0 +1,204 @@
+"""Thin ctypes binding of ``libintsgd.so`` (the C ABI declared in ``include/intsgd.h``).
+
+Argument marshalling only: every step of the IntSGD path runs in the CUDA kernels.  There is no
+CPU fallback; if the library cannot be loaded, or no CUDA device is present when a context is
+created, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+from pathlib import Path
+
+from . import build as _build
+
+MAX_WORKERS = 64
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_ALIGN = -2
+ERR_CUDA = -3
+ERR_SCALE_NONFINITE = -4
+ERR_UNSUPPORTED = -5
+
+GRAD_F32, GRAD_BF16 = 0, 1
+PAYLOAD_I32, PAYLOAD_I8 = 0, 1
+ROUND_RANDOM, ROUND_NEAREST = 0, 1
+MODE_EXACT, MODE_TWO_KERNEL, MODE_FUSED = 0, 1, 2
+
+EXPORTS = [
+    "intsgd_create", "intsgd_destroy", "intsgd_scale", "intsgd_sqdiff", "intsgd_encode",
+    "intsgd_aggregate", "intsgd_step", "intsgd_step_host", "intsgd_get_stats", "intsgd_get_state",
+    "intsgd_set_state", "intsgd_set_launch", "intsgd_launch_count", "intsgd_last_error",
+]
+
+
+class Config(C.Structure):
+    _fields_ = [("n", C.c_int32), ("grad_dtype", C.c_int32), ("d", C.c_int64),
+                ("payload_dtype", C.c_int32), ("rounding", C.c_int32), ("beta", C.c_double),
+                ("eps", C.c_double), ("seed", C.c_uint64), ("clip_limit", C.c_int64),
+                ("device", C.c_int32), ("reserved", C.c_int32)]
+
+
+class State(C.Structure):
+    _fields_ = [("r", C.c_double), ("dx2", C.c_double), ("alpha", C.c_float), ("c", C.c_float),
+                ("step", C.c_uint32), ("status", C.c_int32)]
+
+
+class Stats(C.Structure):
+    _fields_ = [("state", State), ("clip_count", C.c_uint64 * MAX_WORKERS), ("nonfinite", C.c_uint64),
+                ("agg_overflow", C.c_uint64), ("max_abs_agg", C.c_int32), ("reserved", C.c_int32)]
+
+
+class IntSGDError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"intsgd error {code}: {message}")
+        self.code = code
+
+
+_lib = None
+
+
+def library_path() -> Path:
+    return _build.LIB
+
+
+def load() -> C.CDLL:
+    """Load ``libintsgd.so`` (building it with nvcc first if it is absent)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if not path.exists():
+        _build.build()
+    lib = C.CDLL(str(path))
+    vp, i32, i64, f64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_double, C.c_float
+    lib.intsgd_create.argtypes = [C.POINTER(vp), C.POINTER(Config)]
+    lib.intsgd_destroy.argtypes = [vp]
+    lib.intsgd_scale.argtypes = [vp, f64, f64, vp]
+    lib.intsgd_sqdiff.argtypes = [vp, vp, vp, vp]
+    lib.intsgd_encode.argtypes = [vp, i32, vp, vp, f32, vp]
+    lib.intsgd_aggregate.argtypes = [vp, C.POINTER(vp), vp, vp, vp]
+    lib.intsgd_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, vp, f64, i32, vp]
+    lib.intsgd_step_host.argtypes = [vp, C.POINTER(vp), vp, vp, f64, i32, vp]
+    lib.intsgd_get_stats.argtypes = [vp, C.POINTER(Stats)]
+    lib.intsgd_get_state.argtypes = [vp, C.POINTER(State)]
+    lib.intsgd_set_state.argtypes = [vp, C.POINTER(State)]
+    lib.intsgd_set_launch.argtypes = [vp, i32, i32]
+    lib.intsgd_launch_count.argtypes = [vp]
+    lib.intsgd_launch_count.restype = i64
+    lib.intsgd_last_error.argtypes = [vp]
+    lib.intsgd_last_error.restype = C.c_char_p
+    for name in EXPORTS:
+        if name not in ("intsgd_launch_count", "intsgd_last_error"):
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _addr(t) -> int | None:
+    """Device (or host) address of a torch tensor / numpy array / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    if hasattr(t, "ctypes"):
+        return t.ctypes.data
+    raise TypeError(f"cannot take the address of {type(t)}")
+
+
+def _ptr_array(seq):
+    return (C.c_void_p * len(seq))(*[_addr(t) for t in seq])
+
+
+class IntSGD:
+    """One IntSGD context.  Method names and arguments mirror the C ABI one to one."""
+
+    def __init__(self, n, d, *, grad_dtype=GRAD_F32, payload_dtype=PAYLOAD_I32,
+                 rounding=ROUND_RANDOM, beta=0.9, eps=1e-8, seed=0, clip_limit=0, device=0):
+        self._lib = load()
+        self.cfg = Config(n=n, grad_dtype=grad_dtype, d=d, payload_dtype=payload_dtype,
+                          rounding=rounding, beta=beta, eps=eps, seed=seed, clip_limit=clip_limit,
+                          device=device, reserved=0)
+        self._ctx = C.c_void_p()
+        rc = self._lib.intsgd_create(C.byref(self._ctx), C.byref(self.cfg))
+        if rc != OK:
+            msg = self._lib.intsgd_last_error(None).decode()
+            self._ctx = C.c_void_p()
+            raise IntSGDError(rc, msg)
+        self.n, self.d = n, d
+
+    # -- lifetime ---------------------------------------------------------------------------
+    def close(self):
+        if getattr(self, "_ctx", None):
+            self._lib.intsgd_destroy(self._ctx)
+            self._ctx = C.c_void_p()
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def _check(self, rc, allow=()):
+        if rc != OK and rc not in allow:
+            raise IntSGDError(rc, self._lib.intsgd_last_error(self._ctx).decode())
+        return rc
+
+    # -- the calls of the C ABI -----------------------------------------------------------------
+    def intsgd_scale(self, eta_k, dx2_override=-1.0, stream=None):
+        self._check(self._lib.intsgd_scale(self._ctx, eta_k, dx2_override, stream))
+
+    def intsgd_sqdiff(self, x, x_prev, stream=None):
+        self._check(self._lib.intsgd_sqdiff(self._ctx, _addr(x), _addr(x_prev), stream))
+
+    def intsgd_encode(self, worker, grad, payload, alpha_override=math.nan, stream=None):
+        self._check(self._lib.intsgd_encode(self._ctx, worker, _addr(grad), _addr(payload),
+                                            alpha_override, stream))
+
+    def intsgd_aggregate(self, payloads, x, agg=None, stream=None):
+        self._check(self._lib.intsgd_aggregate(self._ctx, _ptr_array(payloads), _addr(x), _addr(agg), stream))
+
+    def intsgd_step(self, grads, x, agg=None, *, eta_k, mode=MODE_FUSED, payload_scratch=None, stream=None):
+        scratch = _ptr_array(payload_scratch) if payload_scratch is not None else None
+        self._check(self._lib.intsgd_step(self._ctx, _ptr_array(grads), scratch, _addr(x), _addr(agg),
+                                          eta_k, mode, stream))
+
+    def intsgd_step_host(self, host_grads, host_x, host_agg=None, *, eta_k, mode=MODE_FUSED, stream=None):
+        self._check(self._lib.intsgd_step_host(self._ctx, _ptr_array(host_grads), _addr(host_x),
+                                               _addr(host_agg), eta_k, mode, stream))
+
+    def intsgd_get_stats(self, allow_nonfinite=False) -> dict:
+        s = Stats()
+        rc = self._check(self._lib.intsgd_get_stats(self._ctx, C.byref(s)),
+                         allow=(ERR_SCALE_NONFINITE,) if allow_nonfinite else ())
+        st = s.state
+        return dict(rc=rc, r=st.r, dx2=st.dx2, alpha=st.alpha, c=st.c, step=st.step, status=st.status,
+                    clip_count=[int(v) for v in s.clip_count[: self.n]], nonfinite=int(s.nonfinite),
+                    agg_overflow=int(s.agg_overflow), max_abs_agg=int(s.max_abs_agg))
+
+    def intsgd_get_state(self) -> State:
+        st = State()
+        self._check(self._lib.intsgd_get_state(self._ctx, C.byref(st)), allow=(ERR_SCALE_NONFINITE,))
+        return st
+
+    def intsgd_set_state(self, *, r, dx2, alpha, c, step, status=OK):
+        st = State(r=r, dx2=dx2, alpha=alpha, c=c, step=step, status=status)
+        self._check(self._lib.intsgd_set_state(self._ctx, C.byref(st)))
+
+    def intsgd_set_launch(self, threads_per_block=0, blocks_per_sm=0):
+        self._check(self._lib.intsgd_set_launch(self._ctx, threads_per_block, blocks_per_sm))
+
+    def intsgd_launch_count(self) -> int:
+        return int(self._lib.intsgd_launch_count(self._ctx))
+
+    def intsgd_last_error(self) -> str:
+        return self._lib.intsgd_last_error(self._ctx).decode()

@@ -1,0 +1,523 @@
+// Host side of the IntSGD step library: argument checks, launch shapes, the C ABI of intsgd.h.
+// Every step of the path runs in the kernels of intsgd_kernels.cuh; there is no CPU fallback.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <limits>
+#include <new>
+
+#include "intsgd_kernels.cuh"
+
+using namespace intsgd;
+
+struct intsgd_ctx {
+    intsgd_config cfg;
+    int64_t L;            // clip limit as an integer
+    float Lf;             // largest fp32 <= L
+    PhiloxKeys keys;
+    DevState* d_state;
+    double* d_partials;
+    int max_grid;
+    int sm_count;
+    int threads;
+    int blocks_per_sm;
+    cudaStream_t last_stream;
+    int64_t launches;
+    // device staging for intsgd_step_host (allocated on first use)
+    void* stage_grads[INTSGD_MAX_WORKERS];
+    float* stage_x;
+    int32_t* stage_agg;
+    char err[256];
+};
+
+namespace {
+
+thread_local char g_create_err[256] = "";
+
+constexpr int kDefaultThreads = 256;
+constexpr int kDefaultBlocksPerSm = 8;
+constexpr int kMaxBlocksPerSm = 32;
+
+int fail(intsgd_ctx* ctx, int code, const char* fmt, const char* detail = "") {
+    char* dst = ctx ? ctx->err : g_create_err;
+    std::snprintf(dst, 256, fmt, detail);
+    return code;
+}
+
+#define CUDA_TRY(ctx, expr)                                                                  \
+    do {                                                                                     \
+        cudaError_t e_ = (expr);                                                             \
+        if (e_ != cudaSuccess) return fail((ctx), INTSGD_ERR_CUDA, #expr ": %s", cudaGetErrorString(e_)); \
+    } while (0)
+
+// Makes the context's device current for the duration of a call and restores the caller's.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t status = cudaSuccess;
+    explicit DeviceGuard(int dev) {
+        status = cudaGetDevice(&prev);
+        if (status == cudaSuccess && prev != dev) {
+            status = cudaSetDevice(dev);
+            switched = (status == cudaSuccess);
+        }
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+size_t grad_elem_size(int dt) { return dt == INTSGD_GRAD_BF16 ? 2 : 4; }
+size_t payload_elem_size(int dt) { return dt == INTSGD_PAYLOAD_I8 ? 1 : 4; }
+
+// Philox key schedule: round r uses key + r * (Weyl constants), modulo 2^32.
+PhiloxKeys make_keys(uint64_t seed) {
+    PhiloxKeys k;
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        k.k0[r] = k0;
+        k.k1[r] = k1;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return k;
+}
+
+float largest_float_not_above(int64_t L) {
+    float f = (float)L;
+    if ((double)f > (double)L) f = std::nextafterf(f, 0.0f);
+    return f;
+}
+
+int grid_for(const intsgd_ctx* ctx, int64_t work_items) {
+    int64_t blocks = (work_items + ctx->threads - 1) / ctx->threads;
+    const int64_t cap = (int64_t)ctx->sm_count * ctx->blocks_per_sm;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+void base_params(const intsgd_ctx* ctx, VecParams& P) {
+    std::memset(&P, 0, sizeof P);
+    P.st = ctx->d_state;
+    P.partials = ctx->d_partials;
+    P.d = ctx->cfg.d;
+    P.n = ctx->cfg.n;
+    P.alpha_override = std::numeric_limits<float>::quiet_NaN();
+    P.Lf = ctx->Lf;
+    P.agg_limit = (ctx->cfg.payload_dtype == INTSGD_PAYLOAD_I8) ? 127 : std::numeric_limits<int32_t>::max();
+    P.keys = ctx->keys;
+}
+
+int check_vector(intsgd_ctx* ctx, const void* p, size_t elem, const char* what, bool* all16) {
+    if (!p) return fail(ctx, INTSGD_ERR_INVALID_ARG, "%s is NULL", what);
+    if (!aligned_to(p, elem)) return fail(ctx, INTSGD_ERR_ALIGN, "%s is not aligned to its element size", what);
+    if (!aligned_to(p, 16)) *all16 = false;
+    return INTSGD_OK;
+}
+
+int after_launch(intsgd_ctx* ctx, const char* what) {
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        std::snprintf(ctx->err, 256, "launch of %s failed: %s", what, cudaGetErrorString(e));
+        return INTSGD_ERR_CUDA;
+    }
+    return INTSGD_OK;
+}
+
+// ---- launchers -------------------------------------------------------------------------
+
+int launch_scale(intsgd_ctx* ctx, double eta, double dx2_override, cudaStream_t s) {
+    if (!(eta > 0.0) || !std::isfinite(eta)) return fail(ctx, INTSGD_ERR_INVALID_ARG, "eta_k must be finite and > 0");
+    if (std::isnan(dx2_override) || std::isinf(dx2_override))
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "dx2_override must be finite (negative = use the state)");
+    const double dd = (double)ctx->cfg.d, dn = (double)ctx->cfg.n;
+    scale_kernel<<<1, 32, 0, s>>>(ctx->d_state, std::sqrt(dd), 2.0 * dn, dn, eta, ctx->cfg.beta, ctx->cfg.eps,
+                                  dx2_override, ctx->cfg.n);
+    return after_launch(ctx, "scale_kernel");
+}
+
+template <int GRAD, int PAY, bool ALIGNED>
+void launch_encode_r(const intsgd_ctx* ctx, const VecParams& P, dim3 grid, cudaStream_t s) {
+    if (ctx->cfg.rounding == INTSGD_ROUND_NEAREST)
+        encode_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
+    else
+        encode_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
+}
+template <int GRAD, int PAY>
+void launch_encode_a(const intsgd_ctx* ctx, const VecParams& P, dim3 grid, bool aligned, cudaStream_t s) {
+    if (aligned) launch_encode_r<GRAD, PAY, true>(ctx, P, grid, s);
+    else launch_encode_r<GRAD, PAY, false>(ctx, P, grid, s);
+}
+int launch_encode(intsgd_ctx* ctx, const VecParams& P, int workers, bool aligned, cudaStream_t s) {
+    dim3 grid((unsigned)grid_for(ctx, (ctx->cfg.d + 3) / 4), (unsigned)workers, 1);
+    // spread the block budget over the workers handled by one launch
+    if (workers > 1) {
+        int per = (ctx->sm_count * ctx->blocks_per_sm + workers - 1) / workers;
+        if (per < 1) per = 1;
+        if ((int)grid.x > per) grid.x = (unsigned)per;
+    }
+    const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16, i8 = ctx->cfg.payload_dtype == INTSGD_PAYLOAD_I8;
+    if (!bf16 && !i8) launch_encode_a<INTSGD_GRAD_F32, INTSGD_PAYLOAD_I32>(ctx, P, grid, aligned, s);
+    else if (!bf16 && i8) launch_encode_a<INTSGD_GRAD_F32, INTSGD_PAYLOAD_I8>(ctx, P, grid, aligned, s);
+    else if (bf16 && !i8) launch_encode_a<INTSGD_GRAD_BF16, INTSGD_PAYLOAD_I32>(ctx, P, grid, aligned, s);
+    else launch_encode_a<INTSGD_GRAD_BF16, INTSGD_PAYLOAD_I8>(ctx, P, grid, aligned, s);
+    return after_launch(ctx, "encode_kernel");
+}
+
+int launch_aggregate(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
+    const bool i8 = ctx->cfg.payload_dtype == INTSGD_PAYLOAD_I8;
+    const int64_t items = (i8 && aligned) ? (ctx->cfg.d + 15) / 16 : (i8 ? ctx->cfg.d : (ctx->cfg.d + 3) / 4);
+    const int grid = grid_for(ctx, items);
+    if (!i8 && aligned) aggregate_kernel<INTSGD_PAYLOAD_I32, true><<<grid, ctx->threads, 0, s>>>(P);
+    else if (!i8) aggregate_kernel<INTSGD_PAYLOAD_I32, false><<<grid, ctx->threads, 0, s>>>(P);
+    else if (aligned) aggregate_kernel<INTSGD_PAYLOAD_I8, true><<<grid, ctx->threads, 0, s>>>(P);
+    else aggregate_kernel<INTSGD_PAYLOAD_I8, false><<<grid, ctx->threads, 0, s>>>(P);
+    return after_launch(ctx, "aggregate_kernel");
+}
+
+template <int GRAD, bool ALIGNED>
+void launch_fused_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStream_t s) {
+    if (ctx->cfg.rounding == INTSGD_ROUND_NEAREST)
+        fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
+    else
+        fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
+}
+int launch_fused(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
+    const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
+    const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
+    if (!bf16 && aligned) launch_fused_r<INTSGD_GRAD_F32, true>(ctx, P, grid, s);
+    else if (!bf16) launch_fused_r<INTSGD_GRAD_F32, false>(ctx, P, grid, s);
+    else if (aligned) launch_fused_r<INTSGD_GRAD_BF16, true>(ctx, P, grid, s);
+    else launch_fused_r<INTSGD_GRAD_BF16, false>(ctx, P, grid, s);
+    return after_launch(ctx, "fused_step_kernel");
+}
+
+int launch_exact(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
+    const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
+    const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
+    if (!bf16 && aligned) exact_step_kernel<INTSGD_GRAD_F32, true><<<grid, ctx->threads, 0, s>>>(P);
+    else if (!bf16) exact_step_kernel<INTSGD_GRAD_F32, false><<<grid, ctx->threads, 0, s>>>(P);
+    else if (aligned) exact_step_kernel<INTSGD_GRAD_BF16, true><<<grid, ctx->threads, 0, s>>>(P);
+    else exact_step_kernel<INTSGD_GRAD_BF16, false><<<grid, ctx->threads, 0, s>>>(P);
+    return after_launch(ctx, "exact_step_kernel");
+}
+
+int read_state_block(intsgd_ctx* ctx, DevState* host) {
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->last_stream));
+    CUDA_TRY(ctx, cudaMemcpy(host, ctx->d_state, sizeof(DevState), cudaMemcpyDeviceToHost));
+    return INTSGD_OK;
+}
+
+void free_staging(intsgd_ctx* ctx) {
+    for (int i = 0; i < INTSGD_MAX_WORKERS; ++i) {
+        if (ctx->stage_grads[i]) cudaFree(ctx->stage_grads[i]);
+        ctx->stage_grads[i] = nullptr;
+    }
+    if (ctx->stage_x) cudaFree(ctx->stage_x);
+    if (ctx->stage_agg) cudaFree(ctx->stage_agg);
+    ctx->stage_x = nullptr;
+    ctx->stage_agg = nullptr;
+}
+
+}  // namespace
+
+// ======================================================================================
+// C ABI
+// ======================================================================================
+extern "C" {
+
+int intsgd_create(intsgd_ctx** out, const intsgd_config* cfg) {
+    g_create_err[0] = 0;
+    if (!out || !cfg) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "intsgd_create: NULL argument");
+    *out = nullptr;
+    if (cfg->n < 1 || cfg->n > INTSGD_MAX_WORKERS) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "n must be in 1..64");
+    if (cfg->d < 1 || cfg->d > ((int64_t)1 << 40)) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "d must be in 1..2^40");
+    if (cfg->grad_dtype != INTSGD_GRAD_F32 && cfg->grad_dtype != INTSGD_GRAD_BF16)
+        return fail(nullptr, INTSGD_ERR_INVALID_ARG, "bad grad_dtype");
+    if (cfg->payload_dtype != INTSGD_PAYLOAD_I32 && cfg->payload_dtype != INTSGD_PAYLOAD_I8)
+        return fail(nullptr, INTSGD_ERR_INVALID_ARG, "bad payload_dtype");
+    if (cfg->rounding != INTSGD_ROUND_RANDOM && cfg->rounding != INTSGD_ROUND_NEAREST)
+        return fail(nullptr, INTSGD_ERR_INVALID_ARG, "bad rounding");
+    if (!(cfg->beta >= 0.0 && cfg->beta < 1.0)) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "beta must be in [0, 1)");
+    if (!(cfg->eps >= 0.0) || !std::isfinite(cfg->eps)) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "eps must be finite and >= 0");
+    if (cfg->reserved != 0) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "reserved must be 0");
+    const int64_t int32_max = std::numeric_limits<int32_t>::max();
+    int64_t L = cfg->clip_limit;
+    if (L == 0) L = (cfg->payload_dtype == INTSGD_PAYLOAD_I8) ? 127 : int32_max / cfg->n;
+    if (L < 1) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "clip_limit must be positive (0 = default)");
+    if (cfg->payload_dtype == INTSGD_PAYLOAD_I8 && L > 127) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "int8 payload needs clip_limit <= 127");
+    if (L > int32_max / cfg->n) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "n * clip_limit must fit int32");
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+        cudaGetLastError();
+        return fail(nullptr, INTSGD_ERR_CUDA, "no CUDA device: this library has no CPU path");
+    }
+    if (cfg->device < 0 || cfg->device >= ndev) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "device ordinal out of range");
+
+    intsgd_ctx* ctx = new (std::nothrow) intsgd_ctx();
+    if (!ctx) return fail(nullptr, INTSGD_ERR_CUDA, "out of host memory");
+    std::memset(ctx, 0, sizeof *ctx);
+    ctx->cfg = *cfg;
+    ctx->L = L;
+    ctx->Lf = largest_float_not_above(L);
+    ctx->keys = make_keys(cfg->seed);
+    ctx->threads = kDefaultThreads;
+    ctx->blocks_per_sm = kDefaultBlocksPerSm;
+
+    DeviceGuard guard(cfg->device);
+    cudaError_t e = guard.status;
+    cudaDeviceProp prop;
+    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, cfg->device);
+    if (e == cudaSuccess) {
+        ctx->sm_count = prop.multiProcessorCount;
+        ctx->max_grid = ctx->sm_count * kMaxBlocksPerSm;
+        e = cudaMalloc(&ctx->d_state, sizeof(DevState));
+    }
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_partials, sizeof(double) * ctx->max_grid);
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_state, 0, sizeof(DevState));
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_partials, 0, sizeof(double) * ctx->max_grid);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        std::snprintf(g_create_err, 256, "intsgd_create: %s", cudaGetErrorString(e));
+        if (ctx->d_state) cudaFree(ctx->d_state);
+        if (ctx->d_partials) cudaFree(ctx->d_partials);
+        delete ctx;
+        return INTSGD_ERR_CUDA;
+    }
+    *out = ctx;
+    return INTSGD_OK;
+}
+
+int intsgd_destroy(intsgd_ctx* ctx) {
+    if (!ctx) return INTSGD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    free_staging(ctx);
+    cudaFree(ctx->d_state);
+    cudaFree(ctx->d_partials);
+    delete ctx;
+    return INTSGD_OK;
+}
+
+int intsgd_scale(intsgd_ctx* ctx, double eta_k, double dx2_override, void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    ctx->last_stream = (cudaStream_t)stream;
+    return launch_scale(ctx, eta_k, dx2_override, (cudaStream_t)stream);
+}
+
+int intsgd_sqdiff(intsgd_ctx* ctx, const float* x, const float* x_prev, void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    bool al = true;
+    int rc;
+    if ((rc = check_vector(ctx, x, 4, "x", &al)) != INTSGD_OK) return rc;
+    if ((rc = check_vector(ctx, x_prev, 4, "x_prev", &al)) != INTSGD_OK) return rc;
+    VecParams P;
+    base_params(ctx, P);
+    P.x = const_cast<float*>(x);
+    P.x_prev = x_prev;
+    cudaStream_t s = (cudaStream_t)stream;
+    ctx->last_stream = s;
+    const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
+    if (al) sqdiff_kernel<true><<<grid, ctx->threads, 0, s>>>(P);
+    else sqdiff_kernel<false><<<grid, ctx->threads, 0, s>>>(P);
+    return after_launch(ctx, "sqdiff_kernel");
+}
+
+int intsgd_encode(intsgd_ctx* ctx, int32_t worker, const void* grad, void* payload, float alpha_override,
+                  void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (worker < 0 || worker >= ctx->cfg.n) return fail(ctx, INTSGD_ERR_INVALID_ARG, "worker index out of range");
+    if (std::isinf(alpha_override) || alpha_override <= 0.0f)
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "alpha_override must be NaN (use state) or finite and > 0");
+    bool al = true;
+    int rc;
+    if ((rc = check_vector(ctx, grad, grad_elem_size(ctx->cfg.grad_dtype), "grad", &al)) != INTSGD_OK) return rc;
+    if ((rc = check_vector(ctx, payload, payload_elem_size(ctx->cfg.payload_dtype), "payload", &al)) != INTSGD_OK) return rc;
+    VecParams P;
+    base_params(ctx, P);
+    P.in[0] = grad;
+    P.out[0] = payload;
+    P.worker_base = worker;
+    P.alpha_override = alpha_override;
+    ctx->last_stream = (cudaStream_t)stream;
+    return launch_encode(ctx, P, 1, al, (cudaStream_t)stream);
+}
+
+int intsgd_aggregate(intsgd_ctx* ctx, const void* const* payloads, float* x, int32_t* agg, void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!payloads) return fail(ctx, INTSGD_ERR_INVALID_ARG, "payloads is NULL");
+    bool al = true;
+    int rc;
+    VecParams P;
+    base_params(ctx, P);
+    for (int i = 0; i < ctx->cfg.n; ++i) {
+        if ((rc = check_vector(ctx, payloads[i], payload_elem_size(ctx->cfg.payload_dtype), "payloads[i]", &al)) != INTSGD_OK) return rc;
+        P.in[i] = payloads[i];
+    }
+    if ((rc = check_vector(ctx, x, 4, "x", &al)) != INTSGD_OK) return rc;
+    if (agg && (rc = check_vector(ctx, agg, 4, "agg", &al)) != INTSGD_OK) return rc;
+    P.x = x;
+    P.agg = agg;
+    ctx->last_stream = (cudaStream_t)stream;
+    return launch_aggregate(ctx, P, al, (cudaStream_t)stream);
+}
+
+int intsgd_step(intsgd_ctx* ctx, const void* const* grads, void* const* payload_scratch, float* x, int32_t* agg,
+                double eta_k, int32_t mode, void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (mode != INTSGD_MODE_EXACT && mode != INTSGD_MODE_TWO_KERNEL && mode != INTSGD_MODE_FUSED)
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "bad mode");
+    if (!grads) return fail(ctx, INTSGD_ERR_INVALID_ARG, "grads is NULL");
+    if (mode == INTSGD_MODE_TWO_KERNEL && !payload_scratch)
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "TWO_KERNEL mode needs payload_scratch");
+    if (!(eta_k > 0.0) || !std::isfinite(eta_k)) return fail(ctx, INTSGD_ERR_INVALID_ARG, "eta_k must be finite and > 0");
+    cudaStream_t s = (cudaStream_t)stream;
+    bool al = true;
+    int rc;
+    VecParams P;
+    base_params(ctx, P);
+    for (int i = 0; i < ctx->cfg.n; ++i) {
+        if ((rc = check_vector(ctx, grads[i], grad_elem_size(ctx->cfg.grad_dtype), "grads[i]", &al)) != INTSGD_OK) return rc;
+        P.in[i] = grads[i];
+    }
+    if ((rc = check_vector(ctx, x, 4, "x", &al)) != INTSGD_OK) return rc;
+    if (agg && (rc = check_vector(ctx, agg, 4, "agg", &al)) != INTSGD_OK) return rc;
+    P.x = x;
+    P.agg = agg;
+    ctx->last_stream = s;
+
+    if (mode == INTSGD_MODE_EXACT) {
+        P.c_exact = (float)(eta_k / (double)ctx->cfg.n);
+        P.agg = nullptr;
+        return launch_exact(ctx, P, al, s);
+    }
+    if (mode == INTSGD_MODE_FUSED) {
+        if ((rc = launch_scale(ctx, eta_k, -1.0, s)) != INTSGD_OK) return rc;
+        return launch_fused(ctx, P, al, s);
+    }
+    // TWO_KERNEL: the payload buffers' alignment decides the encode stores and aggregate loads.
+    bool al_enc = al, al_agg = true;
+    if (!aligned_to(x, 16) || (agg && !aligned_to(agg, 16))) al_agg = false;
+    for (int i = 0; i < ctx->cfg.n; ++i) {
+        if ((rc = check_vector(ctx, payload_scratch[i], payload_elem_size(ctx->cfg.payload_dtype), "payload_scratch[i]", &al_enc)) != INTSGD_OK) return rc;
+        if (!aligned_to(payload_scratch[i], 16)) al_agg = false;
+        P.out[i] = payload_scratch[i];
+    }
+    if ((rc = launch_scale(ctx, eta_k, -1.0, s)) != INTSGD_OK) return rc;
+    P.worker_base = 0;
+    if ((rc = launch_encode(ctx, P, ctx->cfg.n, al_enc, s)) != INTSGD_OK) return rc;
+    VecParams A;
+    base_params(ctx, A);
+    for (int i = 0; i < ctx->cfg.n; ++i) A.in[i] = payload_scratch[i];
+    A.x = x;
+    A.agg = agg;
+    return launch_aggregate(ctx, A, al_agg, s);
+}
+
+int intsgd_step_host(intsgd_ctx* ctx, const void* const* host_grads, float* host_x, int32_t* host_agg,
+                     double eta_k, int32_t mode, void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!host_grads || !host_x) return fail(ctx, INTSGD_ERR_INVALID_ARG, "host_grads / host_x is NULL");
+    if (mode == INTSGD_MODE_TWO_KERNEL) return fail(ctx, INTSGD_ERR_UNSUPPORTED, "step_host runs EXACT or FUSED");
+    const int n = ctx->cfg.n;
+    const size_t d = (size_t)ctx->cfg.d;
+    const size_t gbytes = d * grad_elem_size(ctx->cfg.grad_dtype);
+    for (int i = 0; i < n; ++i)
+        if (!host_grads[i]) return fail(ctx, INTSGD_ERR_INVALID_ARG, "host_grads[i] is NULL");
+    if (!ctx->stage_x) {
+        for (int i = 0; i < n; ++i) CUDA_TRY(ctx, cudaMalloc(&ctx->stage_grads[i], gbytes));
+        CUDA_TRY(ctx, cudaMalloc(&ctx->stage_x, d * sizeof(float)));
+        CUDA_TRY(ctx, cudaMalloc(&ctx->stage_agg, d * sizeof(int32_t)));
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    for (int i = 0; i < n; ++i)
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->stage_grads[i], host_grads[i], gbytes, cudaMemcpyHostToDevice, s));
+    CUDA_TRY(ctx, cudaMemcpyAsync(ctx->stage_x, host_x, d * sizeof(float), cudaMemcpyHostToDevice, s));
+    const int rc = intsgd_step(ctx, (const void* const*)ctx->stage_grads, nullptr, ctx->stage_x,
+                               host_agg ? ctx->stage_agg : nullptr, eta_k, mode, stream);
+    if (rc != INTSGD_OK) return rc;
+    CUDA_TRY(ctx, cudaMemcpyAsync(host_x, ctx->stage_x, d * sizeof(float), cudaMemcpyDeviceToHost, s));
+    if (host_agg && mode != INTSGD_MODE_EXACT)
+        CUDA_TRY(ctx, cudaMemcpyAsync(host_agg, ctx->stage_agg, d * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(ctx, cudaStreamSynchronize(s));
+    return INTSGD_OK;
+}
+
+int intsgd_get_stats(intsgd_ctx* ctx, intsgd_stats* out) {
+    if (!ctx || !out) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    DevState h;
+    const int rc = read_state_block(ctx, &h);
+    if (rc != INTSGD_OK) return rc;
+    std::memset(out, 0, sizeof *out);
+    out->state.r = h.r;
+    out->state.dx2 = h.dx2;
+    out->state.alpha = h.alpha;
+    out->state.c = h.c;
+    out->state.step = h.step;
+    out->state.status = h.status;
+    for (int i = 0; i < INTSGD_MAX_WORKERS; ++i) out->clip_count[i] = h.clip_count[i];
+    out->nonfinite = h.nonfinite;
+    out->agg_overflow = h.agg_overflow;
+    out->max_abs_agg = h.max_abs_agg;
+    if (h.status == INTSGD_ERR_SCALE_NONFINITE)
+        return fail(ctx, INTSGD_ERR_SCALE_NONFINITE, "alpha_k is not finite and positive (r = 0 with eps = 0?); step not applied");
+    return INTSGD_OK;
+}
+
+int intsgd_get_state(intsgd_ctx* ctx, intsgd_state* out) {
+    if (!ctx || !out) return INTSGD_ERR_INVALID_ARG;
+    intsgd_stats s;
+    const int rc = intsgd_get_stats(ctx, &s);
+    if (rc != INTSGD_OK && rc != INTSGD_ERR_SCALE_NONFINITE) return rc;
+    *out = s.state;
+    return rc;
+}
+
+int intsgd_set_state(intsgd_ctx* ctx, const intsgd_state* in) {
+    if (!ctx || !in) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    DevState h;
+    int rc = read_state_block(ctx, &h);
+    if (rc != INTSGD_OK) return rc;
+    h.r = in->r;
+    h.dx2 = in->dx2;
+    h.alpha = in->alpha;
+    h.c = in->c;
+    h.step = in->step;
+    h.status = in->status;
+    h.ticket = 0;
+    CUDA_TRY(ctx, cudaMemcpy(ctx->d_state, &h, sizeof h, cudaMemcpyHostToDevice));
+    return INTSGD_OK;
+}
+
+int intsgd_set_launch(intsgd_ctx* ctx, int32_t threads_per_block, int32_t blocks_per_sm) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    if (threads_per_block != 0) {
+        if (threads_per_block < 32 || threads_per_block > kMaxThreads || (threads_per_block % 32) != 0)
+            return fail(ctx, INTSGD_ERR_INVALID_ARG, "threads_per_block must be a multiple of 32 in 32..512");
+        ctx->threads = threads_per_block;
+    }
+    if (blocks_per_sm != 0) {
+        if (blocks_per_sm < 1 || blocks_per_sm > kMaxBlocksPerSm)
+            return fail(ctx, INTSGD_ERR_INVALID_ARG, "blocks_per_sm must be in 1..32");
+        ctx->blocks_per_sm = blocks_per_sm;
+    }
+    return INTSGD_OK;
+}
+
+int64_t intsgd_launch_count(const intsgd_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* intsgd_last_error(const intsgd_ctx* ctx) { return ctx ? ctx->err : g_create_err; }
+
+}  // extern "C"

@@ -1,0 +1,285 @@
+// Device-side building blocks of the IntSGD step kernels (sm_100a).
+//
+// Work unit: 4 consecutive coordinates = one Philox4x32-10 block (coordinate j uses word j mod 4
+// of block j / 4), one 16-byte fp32 load per worker.  Every kernel walks units grid-stride, so a
+// warp touches 512 contiguous bytes of each stream per iteration.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "intsgd.h"
+
+namespace intsgd {
+
+typedef unsigned long long u64;
+
+// ----------------------------------------------------------------------------------------
+// Device-resident state.  The first 32 bytes have the layout of intsgd_state.
+// ----------------------------------------------------------------------------------------
+struct DevState {
+    double r;
+    double dx2;
+    float alpha;
+    float c;
+    uint32_t step;
+    int32_t status;
+    u64 clip_count[INTSGD_MAX_WORKERS];
+    u64 nonfinite;
+    u64 agg_overflow;
+    int32_t max_abs_agg;
+    uint32_t ticket;   // blocks that have published their partial in the running reduction
+};
+
+// Philox4x32-10 round keys (key schedule done once on the host: the key is the same for every
+// thread, so the ten (k0, k1) pairs travel as kernel parameters and are read from the constant
+// bank).
+struct PhiloxKeys {
+    uint32_t k0[10];
+    uint32_t k1[10];
+};
+
+struct VecParams {
+    const void* in[INTSGD_MAX_WORKERS];   // gradients (encode / fused / exact) or payloads (aggregate)
+    void* out[INTSGD_MAX_WORKERS];        // payloads (encode)
+    float* x;
+    int32_t* agg;
+    const float* x_prev;                  // sqdiff only
+    DevState* st;
+    double* partials;                     // one slot per block of the grid
+    int64_t d;
+    int32_t n;
+    int32_t worker_base;                  // encode: worker index of blockIdx.y == 0
+    float alpha_override;                 // encode: NaN = take alpha from the state
+    float Lf;                             // clip limit as the largest fp32 <= L
+    float c_exact;                        // exact step: fp32(eta / n)
+    int32_t agg_limit;                    // coordinates with |S| above this count as agg_overflow
+    PhiloxKeys keys;
+};
+
+// ----------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11).  One round: the two 32x32->64 products of
+// counter words 0 and 2 with the round multipliers; new counter =
+// (hi(p1) ^ c1 ^ k0, lo(p1), hi(p0) ^ c3 ^ k1, lo(p0)).
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const PhiloxKeys& K) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ K.k1[r];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// Random words of unit `unit` (coordinates 4*unit .. 4*unit+3) of `worker` at `step`.
+__device__ __forceinline__ uint4 draw_unit(int64_t unit, uint32_t worker, uint32_t step,
+                                           const PhiloxKeys& K) {
+    return philox4x32_10((uint32_t)unit, (uint32_t)((uint64_t)unit >> 32), worker, step, K);
+}
+
+// ----------------------------------------------------------------------------------------
+// Loads and stores.  ALIGNED: every vector pointer of the launch is 16-byte aligned.
+// Gradients and payloads are read once (streaming, evict-first); x is read and rewritten.
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_widen(uint32_t h16) { return __uint_as_float(h16 << 16); }
+
+template <int GRAD>
+__device__ __forceinline__ float grad_at(const void* base, int64_t j) {
+    if (GRAD == INTSGD_GRAD_BF16) return bf16_widen(((const uint16_t*)base)[j]);
+    return ((const float*)base)[j];
+}
+
+template <int GRAD, bool ALIGNED>
+__device__ __forceinline__ float4 load_grad4(const void* base, int64_t unit) {
+    if (GRAD == INTSGD_GRAD_F32) {
+        if (ALIGNED) return __ldcs((const float4*)base + unit);
+        const float* p = (const float*)base + 4 * unit;
+        return make_float4(__ldcs(p), __ldcs(p + 1), __ldcs(p + 2), __ldcs(p + 3));
+    } else {
+        if (ALIGNED) {
+            const uint2 v = __ldcs((const uint2*)base + unit);
+            return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u),
+                               __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+        }
+        const uint16_t* p = (const uint16_t*)base + 4 * unit;
+        return make_float4(bf16_widen(__ldcs(p)), bf16_widen(__ldcs(p + 1)), bf16_widen(__ldcs(p + 2)),
+                           bf16_widen(__ldcs(p + 3)));
+    }
+}
+
+template <bool ALIGNED>
+__device__ __forceinline__ float4 load_f4(const float* base, int64_t unit) {
+    if (ALIGNED) return *((const float4*)base + unit);
+    const float* p = base + 4 * unit;
+    return make_float4(p[0], p[1], p[2], p[3]);
+}
+template <bool ALIGNED>
+__device__ __forceinline__ void store_f4(float* base, int64_t unit, float4 v) {
+    if (ALIGNED) { *((float4*)base + unit) = v; return; }
+    float* p = base + 4 * unit;
+    p[0] = v.x; p[1] = v.y; p[2] = v.z; p[3] = v.w;
+}
+template <bool ALIGNED>
+__device__ __forceinline__ void store_i4(int32_t* base, int64_t unit, int4 v) {
+    if (ALIGNED) { __stcs((int4*)base + unit, v); return; }
+    int32_t* p = base + 4 * unit;
+    __stcs(p, v.x); __stcs(p + 1, v.y); __stcs(p + 2, v.z); __stcs(p + 3, v.w);
+}
+template <bool ALIGNED>
+__device__ __forceinline__ int4 load_i4(const int32_t* base, int64_t unit) {
+    if (ALIGNED) return __ldcs((const int4*)base + unit);
+    const int32_t* p = base + 4 * unit;
+    return make_int4(__ldcs(p), __ldcs(p + 1), __ldcs(p + 2), __ldcs(p + 3));
+}
+
+// ----------------------------------------------------------------------------------------
+// Rounding.  y = fl32(alpha * g).  Random: f = floor(y), p = fl32(y - f),
+// u = (w >> 8) * 2^-24, q = f + [u < p]  (Int(t), Section 2 of the paper).
+// The comparison is done as (float)(w >> 8) < p * 2^24: both scalings are exact.
+// ----------------------------------------------------------------------------------------
+template <int ROUND>
+__device__ __forceinline__ int round_in_range(float y, uint32_t w) {
+    if (ROUND == INTSGD_ROUND_NEAREST) return __float2int_rn(y);
+    const float f = floorf(y);
+    const float p = __fsub_rn(y, f);
+    const float uf = __uint2float_rn(w >> 8);
+    const float pscaled = __fmul_rn(p, 16777216.0f);
+    return __float2int_rz(f) + (uf < pscaled ? 1 : 0);
+}
+
+// Full rule with clipping: values outside [-Lf, Lf] saturate, NaN becomes 0, and the event is
+// counted (Section 5.1: local values are clipped so that the aggregate fits the wire type).
+template <int ROUND>
+__device__ __noinline__ int round_checked(float y, uint32_t w, float Lf, u64* clip_slot, u64* nonfinite_slot) {
+    if (fabsf(y) <= Lf) return round_in_range<ROUND>(y, w);
+    atomicAdd(clip_slot, 1ull);
+    if (!(fabsf(y) <= 3.402823466e+38f)) atomicAdd(nonfinite_slot, 1ull);   // NaN or +-Inf
+    if (y > Lf) return (int)Lf;
+    if (y < -Lf) return -(int)Lf;
+    return 0;   // NaN
+}
+
+// One unit of one worker: scale, round, clip.  The common case (all four values in range) has no
+// clamp and no counter traffic.
+template <int ROUND>
+__device__ __forceinline__ int4 round_unit(float4 g, float alpha, uint4 w, float Lf, u64* clip_slot,
+                                           u64* nonfinite_slot) {
+    const float y0 = __fmul_rn(alpha, g.x), y1 = __fmul_rn(alpha, g.y);
+    const float y2 = __fmul_rn(alpha, g.z), y3 = __fmul_rn(alpha, g.w);
+    const bool in_range = (fabsf(y0) <= Lf) & (fabsf(y1) <= Lf) & (fabsf(y2) <= Lf) & (fabsf(y3) <= Lf);
+    int4 q;
+    if (in_range) {
+        q.x = round_in_range<ROUND>(y0, w.x);
+        q.y = round_in_range<ROUND>(y1, w.y);
+        q.z = round_in_range<ROUND>(y2, w.z);
+        q.w = round_in_range<ROUND>(y3, w.w);
+    } else {
+        q.x = round_checked<ROUND>(y0, w.x, Lf, clip_slot, nonfinite_slot);
+        q.y = round_checked<ROUND>(y1, w.y, Lf, clip_slot, nonfinite_slot);
+        q.z = round_checked<ROUND>(y2, w.z, Lf, clip_slot, nonfinite_slot);
+        q.w = round_checked<ROUND>(y3, w.w, Lf, clip_slot, nonfinite_slot);
+    }
+    return q;
+}
+
+// Decode + update of one coordinate: t = fl32(c * float(S)); x_new = fl32(x - t); the squared
+// fp32 step length goes to an fp64 accumulator (Algorithm 1: estimator, update, and the argument
+// of the next moving average).
+__device__ __forceinline__ float update_coord(float x_old, int S, float c, double& acc) {
+    const float t = __fmul_rn(c, __int2float_rn(S));
+    const float x_new = __fsub_rn(x_old, t);
+    const float dj = __fsub_rn(x_new, x_old);
+    acc = __fma_rn((double)dj, (double)dj, acc);   // exact product, one rounding: same as mul then add
+    return x_new;
+}
+
+struct ThreadAcc {
+    double dx2;
+    int32_t max_abs;
+    uint32_t overflow;
+};
+
+__device__ __forceinline__ void note_sum(int S, int32_t agg_limit, ThreadAcc& a) {
+    const int m = abs(S);
+    a.max_abs = max(a.max_abs, m);
+    a.overflow += (m > agg_limit) ? 1u : 0u;
+}
+
+// ----------------------------------------------------------------------------------------
+// Grid-wide reduction of the per-thread accumulators with a fixed shape: warp shuffle tree,
+// per-warp slots in shared memory, one fp64 partial per block in global memory; the block that
+// takes the last ticket adds the partials (strided, then the same tree) and writes state.dx2.
+// The result depends only on the launch shape, never on scheduling.
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ double warp_tree(double v) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, off);
+    return v;
+}
+
+__device__ __forceinline__ double block_tree(double v, double* s_warp) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+    v = warp_tree(v);
+    if (lane == 0) s_warp[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+    if (warp == 0) {
+        t = (lane < nwarps) ? s_warp[lane] : 0.0;
+        t = warp_tree(t);
+    }
+    __syncthreads();
+    return t;   // valid in thread 0
+}
+
+__device__ __forceinline__ void grid_finalize(const ThreadAcc& a, DevState* st, double* partials,
+                                              bool advance_step) {
+    __shared__ double s_warp[32];
+    __shared__ bool s_last;
+    const int mx = __reduce_max_sync(0xFFFFFFFFu, a.max_abs);
+    const unsigned ov = __reduce_add_sync(0xFFFFFFFFu, a.overflow);
+    if ((threadIdx.x & 31) == 0) {
+        if (mx > 0) atomicMax(&st->max_abs_agg, mx);
+        if (ov) atomicAdd(&st->agg_overflow, (u64)ov);
+    }
+    const double block_sum = block_tree(a.dx2, s_warp);
+    if (threadIdx.x == 0) {
+        __stcg(&partials[blockIdx.x], block_sum);
+        __threadfence();
+        const unsigned t = atomicAdd(&st->ticket, 1u);
+        s_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    double v = 0.0;
+    for (unsigned b = threadIdx.x; b < gridDim.x; b += blockDim.x) v += __ldcg(&partials[b]);
+    const double total = block_tree(v, s_warp);
+    if (threadIdx.x == 0) {
+        st->dx2 = total;
+        if (advance_step) st->step += 1;
+        st->ticket = 0;
+    }
+}
+
+// Per-block clip / non-finite counters live in shared memory (slot i < n: worker i's clipped
+// count, slot INTSGD_MAX_WORKERS: non-finite count) and are flushed once per block.
+__device__ __forceinline__ void counters_init(u64* s_cnt) {
+    for (int t = threadIdx.x; t <= INTSGD_MAX_WORKERS; t += blockDim.x) s_cnt[t] = 0;
+    __syncthreads();
+}
+__device__ __forceinline__ void counters_flush(const u64* s_cnt, DevState* st) {
+    __syncthreads();
+    for (int t = threadIdx.x; t <= INTSGD_MAX_WORKERS; t += blockDim.x) {
+        const u64 v = s_cnt[t];
+        if (v) atomicAdd(t < INTSGD_MAX_WORKERS ? &st->clip_count[t] : &st->nonfinite, v);
+    }
+}
+
+}  // namespace intsgd

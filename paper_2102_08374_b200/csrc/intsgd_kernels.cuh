@@ -1,0 +1,313 @@
+// The IntSGD step kernels (sm_100a).  See intsgd_device.cuh for the unit/stream conventions.
+#pragma once
+
+#include "intsgd_device.cuh"
+
+namespace intsgd {
+
+constexpr int kMaxThreads = 512;
+
+// ----------------------------------------------------------------------------------------
+// Scale: Algorithm 1's moving average and Proposition 2's alpha_k, one thread, fp64 with
+// separately rounded operations.  Also opens a new step: clears the per-step counters.
+// ----------------------------------------------------------------------------------------
+__global__ void scale_kernel(DevState* st, double sqrt_d, double two_n, double n_as_double, double eta,
+                             double beta, double eps, double dx2_override, int32_t n) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const double dx2 = (dx2_override >= 0.0) ? dx2_override : st->dx2;
+    const double a = __dmul_rn(beta, st->r);
+    const double b = __dmul_rn(__dsub_rn(1.0, beta), dx2);
+    const double r = __dadd_rn(a, b);
+    const double two_n_r = __dmul_rn(two_n, r);
+    const double inner = __dadd_rn(__ddiv_rn(two_n_r, __dmul_rn(eta, eta)), __dmul_rn(eps, eps));
+    const double alpha64 = __ddiv_rn(sqrt_d, __dsqrt_rn(inner));
+    const float alpha = __double2float_rn(alpha64);
+    const float c = __double2float_rn(__ddiv_rn(eta, __dmul_rn(n_as_double, (double)alpha)));
+    for (int i = 0; i < n; ++i) st->clip_count[i] = 0;
+    st->nonfinite = 0;
+    st->agg_overflow = 0;
+    st->max_abs_agg = 0;
+    st->ticket = 0;
+    const bool ok = (alpha > 0.0f) && (alpha <= 3.402823466e+38f) && (c > 0.0f) && (c <= 3.402823466e+38f);
+    if (!ok) {
+        st->status = INTSGD_ERR_SCALE_NONFINITE;
+        return;
+    }
+    st->r = r;
+    st->alpha = alpha;
+    st->c = c;
+    st->status = INTSGD_OK;
+}
+
+// ----------------------------------------------------------------------------------------
+// Encode: payload_i = clip(Int(alpha g_i)).  grid = (blocks, workers).
+// ----------------------------------------------------------------------------------------
+template <int PAY>
+__device__ __forceinline__ void store_payload4(void* base, int64_t unit, int4 q, bool aligned) {
+    if (PAY == INTSGD_PAYLOAD_I32) {
+        if (aligned) { __stcs((int4*)base + unit, q); return; }
+        int32_t* p = (int32_t*)base + 4 * unit;
+        __stcs(p, q.x); __stcs(p + 1, q.y); __stcs(p + 2, q.z); __stcs(p + 3, q.w);
+    } else {
+        if (aligned) {
+            const uint32_t packed = (uint32_t)(q.x & 0xFF) | ((uint32_t)(q.y & 0xFF) << 8) |
+                                    ((uint32_t)(q.z & 0xFF) << 16) | ((uint32_t)(q.w & 0xFF) << 24);
+            __stcs((uint32_t*)base + unit, packed);
+            return;
+        }
+        int8_t* p = (int8_t*)base + 4 * unit;
+        p[0] = (int8_t)q.x; p[1] = (int8_t)q.y; p[2] = (int8_t)q.z; p[3] = (int8_t)q.w;
+    }
+}
+
+template <int GRAD, int PAY, bool ALIGNED, int ROUND>
+__global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_constant__ VecParams P) {
+    __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
+    DevState* st = P.st;
+    if (st->status != INTSGD_OK) return;
+    counters_init(s_cnt);
+    const float alpha = (P.alpha_override == P.alpha_override) ? P.alpha_override : st->alpha;
+    const uint32_t step = st->step;
+    const int slot = blockIdx.y;
+    const uint32_t worker = (uint32_t)(P.worker_base + slot);
+    const void* g = P.in[slot];
+    void* out = P.out[slot];
+    u64* clip_slot = &s_cnt[worker];
+    u64* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
+
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
+        const float4 gv = load_grad4<GRAD, ALIGNED>(g, unit);
+        uint4 w = make_uint4(0, 0, 0, 0);
+        if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, worker, step, P.keys);
+        const int4 q = round_unit<ROUND>(gv, alpha, w, P.Lf, clip_slot, nonf_slot);
+        store_payload4<PAY>(out, unit, q, ALIGNED);
+    }
+    const int tail = (int)(P.d & 3);
+    if (tail && blockIdx.x == 0 && threadIdx.x == 0) {
+        uint4 w = make_uint4(0, 0, 0, 0);
+        if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(full, worker, step, P.keys);
+        const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
+        for (int e = 0; e < tail; ++e) {
+            const int64_t j = 4 * full + e;
+            const float y = __fmul_rn(alpha, grad_at<GRAD>(g, j));
+            const int q = round_checked<ROUND>(y, wv[e], P.Lf, clip_slot, nonf_slot);
+            if (PAY == INTSGD_PAYLOAD_I32) ((int32_t*)out)[j] = q;
+            else ((int8_t*)out)[j] = (int8_t)q;
+        }
+    }
+    counters_flush(s_cnt, st);
+}
+
+// ----------------------------------------------------------------------------------------
+// Aggregate + decode + update + next-norm partial, one pass.
+// int32 payloads: one unit (4 coordinates) per thread iteration.
+// int8 payloads : four units (16 coordinates, one 16-byte load per worker) per iteration.
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ void add_bytes(int4& s, uint32_t v) {
+    s.x += (int)(int8_t)(v & 0xFF);
+    s.y += (int)(int8_t)((v >> 8) & 0xFF);
+    s.z += (int)(int8_t)((v >> 16) & 0xFF);
+    s.w += (int)(int8_t)(v >> 24);
+}
+
+template <bool ALIGNED>
+__device__ __forceinline__ void apply_unit(const VecParams& P, int64_t unit, int4 S, float c, ThreadAcc& acc) {
+    const float4 xo = load_f4<ALIGNED>(P.x, unit);
+    float4 xn;
+    xn.x = update_coord(xo.x, S.x, c, acc.dx2);
+    xn.y = update_coord(xo.y, S.y, c, acc.dx2);
+    xn.z = update_coord(xo.z, S.z, c, acc.dx2);
+    xn.w = update_coord(xo.w, S.w, c, acc.dx2);
+    store_f4<ALIGNED>(P.x, unit, xn);
+    if (P.agg) store_i4<ALIGNED>(P.agg, unit, S);
+    note_sum(S.x, P.agg_limit, acc);
+    note_sum(S.y, P.agg_limit, acc);
+    note_sum(S.z, P.agg_limit, acc);
+    note_sum(S.w, P.agg_limit, acc);
+}
+
+__device__ __forceinline__ void apply_coord(const VecParams& P, int64_t j, int S, float c, ThreadAcc& acc) {
+    P.x[j] = update_coord(P.x[j], S, c, acc.dx2);
+    if (P.agg) P.agg[j] = S;
+    note_sum(S, P.agg_limit, acc);
+}
+
+template <int PAY, bool ALIGNED>
+__global__ void __launch_bounds__(kMaxThreads) aggregate_kernel(const __grid_constant__ VecParams P) {
+    DevState* st = P.st;
+    if (st->status != INTSGD_OK) return;
+    const float c = st->c;
+    const int n = P.n;
+    ThreadAcc acc = {0.0, 0, 0u};
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int64_t done;   // coordinates covered by the vector loop
+    if (PAY == INTSGD_PAYLOAD_I32) {
+        const int64_t full = P.d >> 2;
+        for (int64_t unit = first; unit < full; unit += stride) {
+            int4 S = make_int4(0, 0, 0, 0);
+#pragma unroll 4
+            for (int i = 0; i < n; ++i) {
+                const int4 q = load_i4<ALIGNED>((const int32_t*)P.in[i], unit);
+                S.x += q.x; S.y += q.y; S.z += q.z; S.w += q.w;
+            }
+            apply_unit<ALIGNED>(P, unit, S, c, acc);
+        }
+        done = full << 2;
+    } else {
+        const int64_t full16 = ALIGNED ? (P.d >> 4) : 0;
+        for (int64_t u16 = first; u16 < full16; u16 += stride) {
+            int4 S0 = make_int4(0, 0, 0, 0), S1 = S0, S2 = S0, S3 = S0;
+#pragma unroll 4
+            for (int i = 0; i < n; ++i) {
+                const uint4 v = __ldcs((const uint4*)P.in[i] + u16);
+                add_bytes(S0, v.x); add_bytes(S1, v.y); add_bytes(S2, v.z); add_bytes(S3, v.w);
+            }
+            apply_unit<ALIGNED>(P, 4 * u16 + 0, S0, c, acc);
+            apply_unit<ALIGNED>(P, 4 * u16 + 1, S1, c, acc);
+            apply_unit<ALIGNED>(P, 4 * u16 + 2, S2, c, acc);
+            apply_unit<ALIGNED>(P, 4 * u16 + 3, S3, c, acc);
+        }
+        done = full16 << 4;
+        if (!ALIGNED) {   // element-wise path for unaligned int8 payloads
+            for (int64_t j = first; j < P.d; j += stride) {
+                int S = 0;
+                for (int i = 0; i < n; ++i) S += (int)((const int8_t*)P.in[i])[j];
+                apply_coord(P, j, S, c, acc);
+            }
+            done = P.d;
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t j = done; j < P.d; ++j) {
+            int S = 0;
+            for (int i = 0; i < n; ++i)
+                S += (PAY == INTSGD_PAYLOAD_I32) ? ((const int32_t*)P.in[i])[j] : (int)((const int8_t*)P.in[i])[j];
+            apply_coord(P, j, S, c, acc);
+        }
+    }
+    grid_finalize(acc, st, P.partials, true);
+}
+
+// ----------------------------------------------------------------------------------------
+// Fused step: encode -> integer sum -> decode -> update -> next-norm partial.  Each thread owns
+// a unit, walks the n gradient streams, rounds in registers and keeps the int32 sums in
+// registers; payloads never reach memory.
+// ----------------------------------------------------------------------------------------
+template <int GRAD, bool ALIGNED, int ROUND>
+__global__ void __launch_bounds__(kMaxThreads) fused_step_kernel(const __grid_constant__ VecParams P) {
+    __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
+    DevState* st = P.st;
+    if (st->status != INTSGD_OK) return;
+    counters_init(s_cnt);
+    const float alpha = st->alpha, c = st->c;
+    const uint32_t step = st->step;
+    const int n = P.n;
+    u64* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
+    ThreadAcc acc = {0.0, 0, 0u};
+
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
+        int4 S = make_int4(0, 0, 0, 0);
+#pragma unroll 4
+        for (int i = 0; i < n; ++i) {
+            const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, (uint32_t)i, step, P.keys);
+            const int4 q = round_unit<ROUND>(gv, alpha, w, P.Lf, &s_cnt[i], nonf_slot);
+            S.x += q.x; S.y += q.y; S.z += q.z; S.w += q.w;
+        }
+        apply_unit<ALIGNED>(P, unit, S, c, acc);
+    }
+    const int tail = (int)(P.d & 3);
+    if (tail && blockIdx.x == 0 && threadIdx.x == 0) {
+        int S[4] = {0, 0, 0, 0};
+        for (int i = 0; i < n; ++i) {
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(full, (uint32_t)i, step, P.keys);
+            const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
+            for (int e = 0; e < tail; ++e) {
+                const float y = __fmul_rn(alpha, grad_at<GRAD>(P.in[i], 4 * full + e));
+                S[e] += round_checked<ROUND>(y, wv[e], P.Lf, &s_cnt[i], nonf_slot);
+            }
+        }
+        for (int e = 0; e < tail; ++e) apply_coord(P, 4 * full + e, S[e], c, acc);
+    }
+    counters_flush(s_cnt, st);
+    grid_finalize(acc, st, P.partials, true);
+}
+
+// ----------------------------------------------------------------------------------------
+// Exact first step (Algorithm 1, Init line): x <- x - fl32(eta/n) * (((g_0 + g_1) + ...) + g_{n-1}).
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ float exact_coord(float x_old, float m, float c0, double& acc) {
+    const float t = __fmul_rn(c0, m);
+    const float x_new = __fsub_rn(x_old, t);
+    const float dj = __fsub_rn(x_new, x_old);
+    acc = __fma_rn((double)dj, (double)dj, acc);
+    return x_new;
+}
+
+template <int GRAD, bool ALIGNED>
+__global__ void __launch_bounds__(kMaxThreads) exact_step_kernel(const __grid_constant__ VecParams P) {
+    const int n = P.n;
+    const float c0 = P.c_exact;
+    ThreadAcc acc = {0.0, 0, 0u};
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
+        float4 m = load_grad4<GRAD, ALIGNED>(P.in[0], unit);
+#pragma unroll 4
+        for (int i = 1; i < n; ++i) {
+            const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
+            m.x = __fadd_rn(m.x, gv.x); m.y = __fadd_rn(m.y, gv.y);
+            m.z = __fadd_rn(m.z, gv.z); m.w = __fadd_rn(m.w, gv.w);
+        }
+        const float4 xo = load_f4<ALIGNED>(P.x, unit);
+        float4 xn;
+        xn.x = exact_coord(xo.x, m.x, c0, acc.dx2);
+        xn.y = exact_coord(xo.y, m.y, c0, acc.dx2);
+        xn.z = exact_coord(xo.z, m.z, c0, acc.dx2);
+        xn.w = exact_coord(xo.w, m.w, c0, acc.dx2);
+        store_f4<ALIGNED>(P.x, unit, xn);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t j = full << 2; j < P.d; ++j) {
+            float m = grad_at<GRAD>(P.in[0], j);
+            for (int i = 1; i < n; ++i) m = __fadd_rn(m, grad_at<GRAD>(P.in[i], j));
+            P.x[j] = exact_coord(P.x[j], m, c0, acc.dx2);
+        }
+    }
+    grid_finalize(acc, P.st, P.partials, true);
+}
+
+// ----------------------------------------------------------------------------------------
+// state.dx2 = ||x - x_prev||^2 (fp32 differences, fp64 sum).
+// ----------------------------------------------------------------------------------------
+template <bool ALIGNED>
+__global__ void __launch_bounds__(kMaxThreads) sqdiff_kernel(const __grid_constant__ VecParams P) {
+    ThreadAcc acc = {0.0, 0, 0u};
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
+        const float4 a = load_f4<ALIGNED>(P.x, unit), b = load_f4<ALIGNED>(P.x_prev, unit);
+        const float d0 = __fsub_rn(a.x, b.x), d1 = __fsub_rn(a.y, b.y);
+        const float d2 = __fsub_rn(a.z, b.z), d3 = __fsub_rn(a.w, b.w);
+        acc.dx2 = __fma_rn((double)d0, (double)d0, acc.dx2);
+        acc.dx2 = __fma_rn((double)d1, (double)d1, acc.dx2);
+        acc.dx2 = __fma_rn((double)d2, (double)d2, acc.dx2);
+        acc.dx2 = __fma_rn((double)d3, (double)d3, acc.dx2);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t j = full << 2; j < P.d; ++j) {
+            const float dj = __fsub_rn(P.x[j], P.x_prev[j]);
+            acc.dx2 = __fma_rn((double)dj, (double)dj, acc.dx2);
+        }
+    }
+    grid_finalize(acc, P.st, P.partials, false);
+}
+
+}  // namespace intsgd

@@ -1,0 +1,153 @@
+"""GPU parity of whole IntSGD steps (exact first step, two-kernel and fused paths) with the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2102_08374_b200 as pkg
+from paper_2102_08374_b200 import synth
+
+from helpers import LockStep, check_window, dev, rel_close, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("mode", [pkg.MODE_FUSED, pkg.MODE_TWO_KERNEL])
+@pytest.mark.parametrize("grad_dtype,payload_dtype", [(pkg.GRAD_F32, pkg.PAYLOAD_I32), (pkg.GRAD_F32, pkg.PAYLOAD_I8),
+                                                      (pkg.GRAD_BF16, pkg.PAYLOAD_I8), (pkg.GRAD_BF16, pkg.PAYLOAD_I32)])
+@pytest.mark.parametrize("rounding", [pkg.ROUND_RANDOM, pkg.ROUND_NEAREST])
+def test_multi_step_lockstep(mode, grad_dtype, payload_dtype, rounding):
+    """Several tiles and a ragged tail: d = 5 * 2^16 + 3 spans many blocks and leaves 3 coordinates."""
+    n, d, eta = 6, 5 * (1 << 16) + 3, 0.1
+    rng = np.random.default_rng(21)
+
+    def grads():
+        out = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
+        out[2][rng.integers(0, d, 50)] *= 300.0     # a few outliers: exercises clipping on the int8 wire
+        return [synth.to_bf16_bits(g) for g in out] if grad_dtype == pkg.GRAD_BF16 else out
+
+    ls = LockStep(n, d, grad_dtype=grad_dtype, payload_dtype=payload_dtype, rounding=rounding, seed=99,
+                  x0=rng.normal(0, 1, d).astype(np.float32))
+    try:
+        ls.exact(grads(), eta)
+        clipped = 0
+        for k in range(5):
+            st, ref = ls.step(grads(), eta, mode=mode)
+            clipped += sum(st["clip_count"])
+        if payload_dtype == pkg.PAYLOAD_I8:
+            assert clipped > 0
+    finally:
+        ls.close()
+
+
+def test_two_kernel_payloads_match_the_oracle():
+    n, d, eta, seed = 4, (1 << 17) + 1, 0.2, 1234
+    rng = np.random.default_rng(3)
+    for payload_dtype in (pkg.PAYLOAD_I32, pkg.PAYLOAD_I8):
+        ls = LockStep(n, d, payload_dtype=payload_dtype, seed=seed, x0=rng.normal(0, 1, d).astype(np.float32))
+        try:
+            g = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
+            ls.exact(g, eta)
+            g = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
+            st, ref = ls.step(g, eta, mode=pkg.MODE_TWO_KERNEL)
+            for i in range(n):
+                want, _, _ = oracle.encode(g[i], np.float32(st["alpha"]), worker=i, step=1, seed=seed, n=n,
+                                           payload_dtype=payload_dtype)
+                assert np.array_equal(ls.last_payloads[i], want)
+        finally:
+            ls.close()
+
+
+@pytest.mark.parametrize("n,d", [(1, 1), (1, 5), (2, 3), (64, 1000), (3, 4), (16, 2)])
+def test_degenerate_shapes(n, d):
+    rng = np.random.default_rng(n * 1000 + d)
+    for mode in (pkg.MODE_FUSED, pkg.MODE_TWO_KERNEL):
+        ls = LockStep(n, d, seed=1, x0=rng.normal(0, 1, d).astype(np.float32))
+        try:
+            ls.exact([rng.normal(0, 1, d).astype(np.float32) for _ in range(n)], 0.1)
+            for _ in range(3):
+                ls.step([rng.normal(0, 1, d).astype(np.float32) for _ in range(n)], 0.1, mode=mode)
+        finally:
+            ls.close()
+
+
+def test_fused_without_aggregate_output():
+    n, d = 3, 70_001
+    rng = np.random.default_rng(5)
+    ls = LockStep(n, d, seed=2, x0=rng.normal(0, 1, d).astype(np.float32))
+    try:
+        ls.exact([rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)], 0.1)
+        ls.step([rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)], 0.1, want_agg=False)
+    finally:
+        ls.close()
+
+
+def test_results_do_not_depend_on_the_launch_shape_and_are_reproducible():
+    n, d, seed = 4, (1 << 19) + 2, 31
+    rng = np.random.default_rng(6)
+    grads = [to_dev(rng.normal(0, 1e-2, d).astype(np.float32)) for _ in range(n)]
+    x0 = rng.normal(0, 1, d).astype(np.float32)
+    outs = []
+    for threads, bps in [(256, 8), (256, 8), (128, 3), (512, 1), (32, 32)]:
+        with pkg.IntSGD(n, d, seed=seed) as lib:
+            lib.intsgd_set_launch(threads, bps)
+            x = to_dev(x0.copy())
+            agg = torch.zeros(d, dtype=torch.int32, device=dev())
+            lib.intsgd_set_state(r=0.0, dx2=2e-3, alpha=0.0, c=0.0, step=1)
+            lib.intsgd_step(grads, x, agg, eta_k=0.1, mode=pkg.MODE_FUSED)
+            st = lib.intsgd_get_stats()
+            outs.append((to_host(x), to_host(agg), st["dx2"], st["max_abs_agg"]))
+    for o in outs[1:]:
+        assert np.array_equal(o[0], outs[0][0]) and np.array_equal(o[1], outs[0][1]) and o[3] == outs[0][3]
+        assert rel_close(o[2], outs[0][2], 1e-13)
+    assert outs[0][2] == outs[1][2]     # same launch shape: bit-identical reduction
+
+
+def test_checkpoint_resume_is_bit_exact():
+    n, d, seed, eta = 3, 50_003, 17, 0.1
+    rng = np.random.default_rng(7)
+    steps = [[to_dev(rng.normal(0, 1e-2, d).astype(np.float32)) for _ in range(n)] for _ in range(10)]
+    x0 = rng.normal(0, 1, d).astype(np.float32)
+
+    def run(lib, x, lo, hi):
+        for k in range(lo, hi):
+            lib.intsgd_step(steps[k], x, None, eta_k=eta, mode=pkg.MODE_EXACT if k == 0 else pkg.MODE_FUSED)
+
+    with pkg.IntSGD(n, d, seed=seed) as a:
+        xa = to_dev(x0.copy())
+        run(a, xa, 0, 10)
+        sa = a.intsgd_get_stats()
+    with pkg.IntSGD(n, d, seed=seed) as b:
+        xb = to_dev(x0.copy())
+        run(b, xb, 0, 5)
+        saved = b.intsgd_get_state()
+        x_saved = xb.clone()
+    with pkg.IntSGD(n, d, seed=seed) as c:
+        c.intsgd_set_state(r=saved.r, dx2=saved.dx2, alpha=saved.alpha, c=saved.c, step=saved.step)
+        run(c, x_saved, 5, 10)
+        sc = c.intsgd_get_stats()
+    assert torch.equal(xa, x_saved)
+    assert (sa["r"], sa["dx2"], sa["alpha"], sa["step"]) == (sc["r"], sc["dx2"], sc["alpha"], sc["step"])
+
+
+def test_step_host_matches_the_device_path():
+    n, d, seed, eta = 4, 300_001, 3, 0.1
+    rng = np.random.default_rng(8)
+    grads = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
+    x0 = rng.normal(0, 1, d).astype(np.float32)
+    with pkg.IntSGD(n, d, seed=seed) as a:
+        xa = to_dev(x0.copy())
+        agg_a = torch.zeros(d, dtype=torch.int32, device=dev())
+        ga = [to_dev(g) for g in grads]
+        a.intsgd_step(ga, xa, None, eta_k=eta, mode=pkg.MODE_EXACT)
+        a.intsgd_step(ga, xa, agg_a, eta_k=eta, mode=pkg.MODE_FUSED)
+        sa = a.intsgd_get_stats()
+    with pkg.IntSGD(n, d, seed=seed) as b:
+        hx = torch.from_numpy(x0.copy()).pin_memory()
+        hg = [torch.from_numpy(g).pin_memory() for g in grads]
+        hagg = torch.zeros(d, dtype=torch.int32).pin_memory()
+        b.intsgd_step_host(hg, hx, None, eta_k=eta, mode=pkg.MODE_EXACT)
+        b.intsgd_step_host(hg, hx, hagg, eta_k=eta, mode=pkg.MODE_FUSED)
+        sb = b.intsgd_get_stats()
+    assert np.array_equal(hx.numpy(), to_host(xa)) and np.array_equal(hagg.numpy(), to_host(agg_a))
+    assert sa["dx2"] == sb["dx2"] and sa["alpha"] == sb["alpha"]
