@@ -47,6 +47,8 @@ extern "C" {
 #define INTSGD_ERR_CUDA             -3   /* a CUDA runtime call failed; see intsgd_last_error */
 #define INTSGD_ERR_SCALE_NONFINITE  -4   /* alpha_k or c_k not finite or not positive; step not applied */
 #define INTSGD_ERR_UNSUPPORTED      -5   /* valid request this build does not implement */
+#define INTSGD_ERR_TIMEOUT          -6   /* a bounded wait inside a kernel gave up; that step's results are
+                                            invalid; sticky until intsgd_set_state */
 
 /* enums (plain ints in the structs) */
 #define INTSGD_GRAD_F32      0
@@ -157,10 +159,16 @@ int intsgd_get_state(intsgd_ctx* ctx, intsgd_state* out);
 /* Overwrite the scalar state (checkpoint resume; tests that impose alpha and c). */
 int intsgd_set_state(intsgd_ctx* ctx, const intsgd_state* in);
 
-/* Tuning knob: threads per block (multiple of 32, <= 1024) and resident blocks per SM used to
+/* Tuning knob: threads per block (multiple of 32, <= 512) and resident blocks per SM used to
  * size the grids of the vector kernels.  0 keeps the built-in value.  Results do not depend on
  * it except the summation order of dx2. */
 int intsgd_set_launch(intsgd_ctx* ctx, int32_t threads_per_block, int32_t blocks_per_sm);
+
+/* Which kernel runs INTSGD_MODE_FUSED: 0 = automatic (the pipelined kernel -- bulk asynchronous copies
+ * into a shared-memory ring -- when every pointer is 16-byte aligned and d <= 2^34, else the direct
+ * kernel), 1 = always the direct kernel, 2 = same as 0.  Both give identical x, aggregate and
+ * counters; dx2 differs only by summation order. */
+int intsgd_set_fused_path(intsgd_ctx* ctx, int32_t path);
 
 /* Number of kernels this library has launched on the context since creation. */
 int64_t intsgd_launch_count(const intsgd_ctx* ctx);

@@ -20,6 +20,7 @@ ERR_ALIGN = -2
 ERR_CUDA = -3
 ERR_SCALE_NONFINITE = -4
 ERR_UNSUPPORTED = -5
+ERR_TIMEOUT = -6
 
 GRAD_F32, GRAD_BF16 = 0, 1
 PAYLOAD_I32, PAYLOAD_I8 = 0, 1
@@ -29,7 +30,7 @@ MODE_EXACT, MODE_TWO_KERNEL, MODE_FUSED = 0, 1, 2
 EXPORTS = [
     "intsgd_create", "intsgd_destroy", "intsgd_scale", "intsgd_sqdiff", "intsgd_encode",
     "intsgd_aggregate", "intsgd_step", "intsgd_step_host", "intsgd_get_stats", "intsgd_get_state",
-    "intsgd_set_state", "intsgd_set_launch", "intsgd_launch_count", "intsgd_last_error",
+    "intsgd_set_state", "intsgd_set_launch", "intsgd_set_fused_path", "intsgd_launch_count", "intsgd_last_error",
 ]
 
 
@@ -85,6 +86,7 @@ def load() -> C.CDLL:
     lib.intsgd_get_state.argtypes = [vp, C.POINTER(State)]
     lib.intsgd_set_state.argtypes = [vp, C.POINTER(State)]
     lib.intsgd_set_launch.argtypes = [vp, i32, i32]
+    lib.intsgd_set_fused_path.argtypes = [vp, i32]
     lib.intsgd_launch_count.argtypes = [vp]
     lib.intsgd_launch_count.restype = i64
     lib.intsgd_last_error.argtypes = [vp]
@@ -196,6 +198,9 @@ class IntSGD:
 
     def intsgd_set_launch(self, threads_per_block=0, blocks_per_sm=0):
         self._check(self._lib.intsgd_set_launch(self._ctx, threads_per_block, blocks_per_sm))
+
+    def intsgd_set_fused_path(self, path: int):
+        self._check(self._lib.intsgd_set_fused_path(self._ctx, path))
 
     def intsgd_launch_count(self) -> int:
         return int(self._lib.intsgd_launch_count(self._ctx))

@@ -7,6 +7,7 @@
 #include <new>
 
 #include "intsgd_kernels.cuh"
+#include "intsgd_pipe.cuh"
 
 using namespace intsgd;
 
@@ -15,6 +16,8 @@ struct intsgd_ctx {
     int64_t L;            // clip limit as an integer
     float Lf;             // largest fp32 <= L
     PhiloxKeys keys;
+    PhiloxWorkerTable tab;
+    int fused_path;       // 0 = automatic, 1 = direct (register) kernel, 2 = pipelined kernel
     DevState* d_state;
     double* d_partials;
     int max_grid;
@@ -83,6 +86,21 @@ PhiloxKeys make_keys(uint64_t seed) {
         k1 += 0xBB67AE85u;
     }
     return k;
+}
+
+// Worker-dependent part of Philox rounds 1-2 for counter (unit, 0, worker, step): see
+// PhiloxWorkerTable.
+PhiloxWorkerTable make_worker_table(const PhiloxKeys& k) {
+    PhiloxWorkerTable t;
+    for (uint32_t i = 0; i < INTSGD_MAX_WORKERS; ++i) {
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)i;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ k.k0[0];
+        const uint64_t q0 = (uint64_t)0xD2511F53u * (uint64_t)n0;
+        t.a[i] = (uint32_t)p1 ^ k.k0[1];
+        t.b[i] = (uint32_t)(q0 >> 32) ^ k.k1[1];
+        t.c[i] = (uint32_t)q0;
+    }
+    return t;
 }
 
 float largest_float_not_above(int64_t L) {
@@ -186,7 +204,61 @@ void launch_fused_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStr
     else
         fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
+
+// Pipelined kernel: kPipeConsumers consumer threads + one producer warp, kPipeGroup worker tiles per
+// stage, kPipeStages stages (192 KiB of shared memory for fp32 gradients), one block per SM.
+constexpr int kPipeConsumers = 512, kPipeGroup = 4, kPipeStages = 6;
+
+template <int GRAD, int ROUND, bool CLAMP>
+cudaError_t launch_pipe_t(const intsgd_ctx* ctx, const PipeParams& PP, cudaStream_t s) {
+    auto kernel = fused_pipe_kernel<GRAD, ROUND, CLAMP, kPipeConsumers, kPipeGroup, kPipeStages, 1>;
+    const int unit_bytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
+    const int smem = kPipeStages * kPipeGroup * kPipeConsumers * unit_bytes;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    int64_t grid = PP.tiles < ctx->sm_count ? PP.tiles : ctx->sm_count;
+    kernel<<<(unsigned)grid, kPipeConsumers + 32, smem, s>>>(PP);
+    return cudaSuccess;
+}
+template <int GRAD, int ROUND>
+cudaError_t launch_pipe_c(const intsgd_ctx* ctx, const PipeParams& PP, bool clamp, cudaStream_t s) {
+    return clamp ? launch_pipe_t<GRAD, ROUND, true>(ctx, PP, s) : launch_pipe_t<GRAD, ROUND, false>(ctx, PP, s);
+}
+
+bool pipe_eligible(const intsgd_ctx* ctx, bool aligned) {
+    const int64_t units = ctx->cfg.d >> 2;
+    return aligned && ctx->cfg.d <= ((int64_t)1 << 34) && units >= 2;
+}
+
+int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
+    PipeParams PP;
+    PP.v = P;
+    PP.tab = ctx->tab;
+    const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
+    int64_t units = ctx->cfg.d >> 2;
+    if (bf16) units &= ~(int64_t)1;   // bulk copies move multiples of 16 bytes
+    PP.units = units;
+    PP.tiles = (units + kPipeConsumers - 1) / kPipeConsumers;
+    // Floors and up-decisions are summed as integer-valued floats: exact while n * (T + 1) <= 2^24.
+    const float t_max = (float)((1 << 24) / ctx->cfg.n - 2);
+    const bool clamp = ctx->Lf <= t_max;   // small limit (int8 wire): clamp in line, no redo for clipping
+    PP.fast_limit = clamp ? 3.402823466e+38f : t_max;
+    const bool nearest = ctx->cfg.rounding == INTSGD_ROUND_NEAREST;
+    cudaError_t e;
+    if (!bf16 && !nearest) e = launch_pipe_c<INTSGD_GRAD_F32, INTSGD_ROUND_RANDOM>(ctx, PP, clamp, s);
+    else if (!bf16) e = launch_pipe_c<INTSGD_GRAD_F32, INTSGD_ROUND_NEAREST>(ctx, PP, clamp, s);
+    else if (!nearest) e = launch_pipe_c<INTSGD_GRAD_BF16, INTSGD_ROUND_RANDOM>(ctx, PP, clamp, s);
+    else e = launch_pipe_c<INTSGD_GRAD_BF16, INTSGD_ROUND_NEAREST>(ctx, PP, clamp, s);
+    if (e != cudaSuccess) {
+        std::snprintf(ctx->err, 256, "fused_pipe_kernel setup failed: %s", cudaGetErrorString(e));
+        return INTSGD_ERR_CUDA;
+    }
+    return after_launch(ctx, "fused_pipe_kernel");
+}
+
 int launch_fused(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
+    const bool want_pipe = ctx->fused_path != 1 && pipe_eligible(ctx, aligned);
+    if (want_pipe) return launch_fused_pipe(ctx, P, s);
     const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
     if (!bf16 && aligned) launch_fused_r<INTSGD_GRAD_F32, true>(ctx, P, grid, s);
@@ -266,6 +338,8 @@ int intsgd_create(intsgd_ctx** out, const intsgd_config* cfg) {
     ctx->L = L;
     ctx->Lf = largest_float_not_above(L);
     ctx->keys = make_keys(cfg->seed);
+    ctx->tab = make_worker_table(ctx->keys);
+    ctx->fused_path = 0;
     ctx->threads = kDefaultThreads;
     ctx->blocks_per_sm = kDefaultBlocksPerSm;
 
@@ -470,6 +544,8 @@ int intsgd_get_stats(intsgd_ctx* ctx, intsgd_stats* out) {
     out->nonfinite = h.nonfinite;
     out->agg_overflow = h.agg_overflow;
     out->max_abs_agg = h.max_abs_agg;
+    if (h.fault)
+        return fail(ctx, INTSGD_ERR_TIMEOUT, "a bounded wait inside a kernel gave up; the results of that step are invalid");
     if (h.status == INTSGD_ERR_SCALE_NONFINITE)
         return fail(ctx, INTSGD_ERR_SCALE_NONFINITE, "alpha_k is not finite and positive (r = 0 with eps = 0?); step not applied");
     return INTSGD_OK;
@@ -497,6 +573,7 @@ int intsgd_set_state(intsgd_ctx* ctx, const intsgd_state* in) {
     h.step = in->step;
     h.status = in->status;
     h.ticket = 0;
+    h.fault = 0;
     CUDA_TRY(ctx, cudaMemcpy(ctx->d_state, &h, sizeof h, cudaMemcpyHostToDevice));
     return INTSGD_OK;
 }
@@ -513,6 +590,13 @@ int intsgd_set_launch(intsgd_ctx* ctx, int32_t threads_per_block, int32_t blocks
             return fail(ctx, INTSGD_ERR_INVALID_ARG, "blocks_per_sm must be in 1..32");
         ctx->blocks_per_sm = blocks_per_sm;
     }
+    return INTSGD_OK;
+}
+
+int intsgd_set_fused_path(intsgd_ctx* ctx, int32_t path) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    if (path < 0 || path > 2) return fail(ctx, INTSGD_ERR_INVALID_ARG, "path must be 0 (auto), 1 (direct) or 2 (pipelined)");
+    ctx->fused_path = path;
     return INTSGD_OK;
 }
 

@@ -29,6 +29,8 @@ struct DevState {
     u64 agg_overflow;
     int32_t max_abs_agg;
     uint32_t ticket;   // blocks that have published their partial in the running reduction
+    int32_t fault;     // sticky: a bounded wait inside a kernel gave up (results of that step are invalid)
+    int32_t pad;
 };
 
 // Philox4x32-10 round keys (key schedule done once on the host: the key is the same for every

@@ -1,0 +1,321 @@
+// Pipelined fused IntSGD step for sm_100a: gradient tiles are staged into shared memory by bulk
+// asynchronous copies (cp.async.bulk, completion counted on mbarriers) issued by one producer
+// thread, while the consumer warps round, sum and update out of shared memory.  The ring of stages
+// keeps ~200 KB of loads in flight per SM independently of the consumers' register use, which is
+// what a 17-stream read at HBM3e speed needs.
+//
+// Layout of one stage: G worker tiles back to back, each kConsumers units of 16 (fp32) or 8 (bf16)
+// bytes; consumer thread c owns unit c of every tile, so shared-memory reads are conflict-free
+// 16-byte (8-byte) accesses and the Philox counter of a thread is fixed for a whole tile.
+//
+// Requirements checked by the host: every pointer 16-byte aligned, d <= 2^34.  Everything else
+// (unaligned pointers, larger d) runs in fused_step_kernel.
+#pragma once
+
+#include "intsgd_device.cuh"
+
+namespace intsgd {
+
+// ---- mbarrier / bulk-copy primitives (inline PTX) -------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+// Bounded wait: gives up after kWaitLimit polls (each poll may itself block for a
+// hardware-defined interval), so a lost completion can never hang the GPU.
+constexpr uint32_t kWaitLimit = 1u << 22;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// Global -> shared bulk copy, completion signalled on an mbarrier of this CTA (no multicast).
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(dst_smem)),
+                 "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+// max(|a|, |b|) up to sign, NaN if either is NaN.
+__device__ __forceinline__ float absmax_nan(float a, float b) {
+    float d;
+    asm("max.NaN.xorsign.abs.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
+// ---- per-unit arithmetic ------------------------------------------------------------------------
+// Fast path of one worker's unit.  Floors and up-decisions are accumulated as integer-valued
+// floats (exact: the host caps the fast-path magnitude T so that n * (T + 1) <= 2^24); `m` tracks
+// max |alpha g| (NaN-propagating) so that anything outside the fast path is redone exactly.
+template <int ROUND, bool CLAMP>
+__device__ __forceinline__ void consume_unit(float4 g, float2 alpha2, uint4 w, float Lf, float2& F01, float2& F23,
+                                             float& m, uint32_t& clipped) {
+    float2 y01 = __fmul2_rn(alpha2, make_float2(g.x, g.y));
+    float2 y23 = __fmul2_rn(alpha2, make_float2(g.z, g.w));
+    m = absmax_nan(m, y01.x); m = absmax_nan(m, y01.y);
+    m = absmax_nan(m, y23.x); m = absmax_nan(m, y23.y);
+    if (CLAMP) {
+        clipped += (fabsf(y01.x) > Lf) + (fabsf(y01.y) > Lf) + (fabsf(y23.x) > Lf) + (fabsf(y23.y) > Lf);
+        y01.x = fminf(fmaxf(y01.x, -Lf), Lf); y01.y = fminf(fmaxf(y01.y, -Lf), Lf);
+        y23.x = fminf(fmaxf(y23.x, -Lf), Lf); y23.y = fminf(fmaxf(y23.y, -Lf), Lf);
+    }
+    if (ROUND == INTSGD_ROUND_NEAREST) {
+        F01 = __fadd2_rn(F01, make_float2(rintf(y01.x), rintf(y01.y)));
+        F23 = __fadd2_rn(F23, make_float2(rintf(y23.x), rintf(y23.y)));
+        return;
+    }
+    const float2 f01 = make_float2(floorf(y01.x), floorf(y01.y));
+    const float2 f23 = make_float2(floorf(y23.x), floorf(y23.y));
+    const float2 neg1 = make_float2(-1.0f, -1.0f), scale = make_float2(16777216.0f, 16777216.0f);
+    const float2 p01 = __fmul2_rn(__ffma2_rn(f01, neg1, y01), scale);   // fl32(y - f) * 2^24, both exact steps
+    const float2 p23 = __fmul2_rn(__ffma2_rn(f23, neg1, y23), scale);
+    const float2 u01 = make_float2(__uint2float_rn(w.x >> 8) < p01.x ? 1.0f : 0.0f,
+                                   __uint2float_rn(w.y >> 8) < p01.y ? 1.0f : 0.0f);
+    const float2 u23 = make_float2(__uint2float_rn(w.z >> 8) < p23.x ? 1.0f : 0.0f,
+                                   __uint2float_rn(w.w >> 8) < p23.y ? 1.0f : 0.0f);
+    F01 = __fadd2_rn(__fadd2_rn(F01, f01), u01);
+    F23 = __fadd2_rn(__fadd2_rn(F23, f23), u23);
+}
+
+// Exact redo of one unit from global memory (rare: a value outside the fast-path range, or a
+// NaN/Inf).  In CLAMP mode the fast path has already counted |y| > Lf, so only NaN adds a clip.
+template <int GRAD, int ROUND, bool CLAMP>
+__device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float alpha, uint32_t step, u64* s_cnt) {
+    int S[4] = {0, 0, 0, 0};
+    for (int i = 0; i < P.n; ++i) {
+        const float4 g = load_grad4<GRAD, true>(P.in[i], unit);
+        uint4 w = make_uint4(0, 0, 0, 0);
+        if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, (uint32_t)i, step, P.keys);
+        const float gv[4] = {g.x, g.y, g.z, g.w};
+        const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
+        for (int e = 0; e < 4; ++e) {
+            const float y = __fmul_rn(alpha, gv[e]);
+            const bool in = fabsf(y) <= P.Lf;
+            if (in) { S[e] += round_in_range<ROUND>(y, wv[e]); continue; }
+            const bool is_nan = (y != y);
+            if (!CLAMP || is_nan) atomicAdd(&s_cnt[i], 1ull);
+            if (!(fabsf(y) <= 3.402823466e+38f)) atomicAdd(&s_cnt[INTSGD_MAX_WORKERS], 1ull);
+            S[e] += is_nan ? 0 : (y > 0.0f ? (int)P.Lf : -(int)P.Lf);
+        }
+    }
+    return make_int4(S[0], S[1], S[2], S[3]);
+}
+
+// Round-1/round-2 Philox values that depend only on (seed, worker) when the high counter word is
+// zero (d <= 2^34): computed on the host once per context.
+struct PhiloxWorkerTable {
+    uint32_t a[INTSGD_MAX_WORKERS];   // lo(M1 * i) ^ k0[1]
+    uint32_t b[INTSGD_MAX_WORKERS];   // hi(M0 * n0) ^ k1[1],  n0 = hi(M1 * i) ^ k0[0]
+    uint32_t c[INTSGD_MAX_WORKERS];   // lo(M0 * n0)
+};
+
+struct PipeParams {
+    VecParams v;
+    PhiloxWorkerTable tab;
+    float fast_limit;   // T: fast path handles |alpha g| <= T
+    int64_t units;      // units covered by the pipeline (the rest is the scalar tail)
+    int64_t tiles;
+};
+
+// Philox4x32-10 for counter (unit, 0, worker, step) with rounds 1-2 folded:
+// per tile and thread: p0 = M0 * unit -> n3 = lo, n2 = hi ^ step ^ k1[0]; p1' = M1 * n2 -> H, m1.
+// per worker: m0 = H ^ a[i], m2 = b[i] ^ n3, m3 = c[i]; then rounds 3..10.
+struct PhiloxThreadPart {
+    uint32_t n3, H, m1;
+};
+__device__ __forceinline__ PhiloxThreadPart philox_thread_part(uint32_t unit_lo, uint32_t step, const PhiloxKeys& K) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)unit_lo;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ step ^ K.k1[0];
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)n2;
+    PhiloxThreadPart t;
+    t.n3 = (uint32_t)p0;
+    t.H = (uint32_t)(p1 >> 32);
+    t.m1 = (uint32_t)p1;
+    return t;
+}
+__device__ __forceinline__ uint4 philox_finish(const PhiloxThreadPart& t, uint32_t a, uint32_t b, uint32_t c,
+                                               const PhiloxKeys& K) {
+    uint32_t c0 = t.H ^ a, c1 = t.m1, c2 = b ^ t.n3, c3 = c;
+#pragma unroll
+    for (int r = 2; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ K.k1[r];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+template <int GRAD>
+__device__ __forceinline__ float4 lds_unit(const unsigned char* tile, int c) {
+    if (GRAD == INTSGD_GRAD_F32) return *reinterpret_cast<const float4*>(tile + 16 * c);
+    const uint2 v = *reinterpret_cast<const uint2*>(tile + 8 * c);
+    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u),
+                       __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+}
+
+// ---- the kernel ----------------------------------------------------------------------------------
+// NC consumer threads + one producer warp.  G worker tiles per stage, NS stages.
+template <int GRAD, int ROUND, bool CLAMP, int NC, int G, int NS, int MINB>
+__global__ void __launch_bounds__(NC + 32, MINB) fused_pipe_kernel(const __grid_constant__ PipeParams PP) {
+    constexpr int kUnitBytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
+    constexpr int kTileBytes = NC * kUnitBytes;
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ uint64_t full_bar[NS], empty_bar[NS];
+    __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
+    __shared__ int s_fault;
+
+    const VecParams& P = PP.v;
+    DevState* st = P.st;
+    if (st->status != INTSGD_OK) return;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], NC);
+        }
+        s_fault = 0;
+        mbar_fence_init();
+    }
+    counters_init(s_cnt);   // includes a __syncthreads()
+
+    const int n = P.n;
+    const int64_t tiles = PP.tiles;
+    ThreadAcc acc = {0.0, 0, 0u};
+    bool ok = true;
+
+    if (threadIdx.x >= NC) {
+        // ------------------------------- producer ---------------------------------------------
+        if (threadIdx.x == NC) {
+            uint32_t it = 0;
+            for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+                const int64_t left = PP.units - tile * NC;
+                const uint32_t bytes = (uint32_t)(left < NC ? left : NC) * kUnitBytes;
+                const size_t offset = (size_t)tile * kTileBytes;
+                for (int g0 = 0; g0 < n; g0 += G, ++it) {
+                    const uint32_t s = it % NS;
+                    if (it >= NS && !mbar_wait(&empty_bar[s], ((it / NS) & 1u) ^ 1u)) { ok = false; break; }
+                    const int gw = (n - g0 < G) ? (n - g0) : G;
+                    mbar_arrive_expect_tx(&full_bar[s], (uint32_t)gw * bytes);
+                    unsigned char* dst = smem + (size_t)s * G * kTileBytes;
+                    for (int w = 0; w < gw; ++w)
+                        bulk_load(dst + w * kTileBytes, (const unsigned char*)P.in[g0 + w] + offset, bytes, &full_bar[s]);
+                }
+            }
+            if (!ok) {
+                // a wait gave up: let every copy still in flight land before this CTA can exit
+                atomicExch(&s_fault, 1);
+                const uint32_t pending = it < NS ? it : NS;
+                for (uint32_t k = 0; k < pending; ++k) {
+                    const uint32_t j = it - 1 - k;
+                    mbar_wait(&full_bar[j % NS], (j / NS) & 1u);
+                }
+            }
+        }
+    } else {
+        // ------------------------------- consumers --------------------------------------------
+        const int c = threadIdx.x;
+        const float alpha = st->alpha, cdec = st->c;
+        const uint32_t step = st->step;
+        const float2 alpha2 = make_float2(alpha, alpha);
+        uint32_t it = 0;
+        for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+            const int64_t unit = tile * NC + c;
+            const bool active = unit < PP.units;
+            float4 xo = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (active) xo = load_f4<true>(P.x, unit);
+            PhiloxThreadPart tp = {0, 0, 0};
+            if (ROUND == INTSGD_ROUND_RANDOM) tp = philox_thread_part((uint32_t)unit, step, P.keys);
+            float2 F01 = make_float2(0.f, 0.f), F23 = F01;
+            float m = 0.0f;
+            for (int g0 = 0; g0 < n; g0 += G, ++it) {
+                const uint32_t s = it % NS;
+                if (!mbar_wait(&full_bar[s], (it / NS) & 1u)) { ok = false; break; }
+                const unsigned char* src = smem + (size_t)s * G * kTileBytes;
+                const int gw = (n - g0 < G) ? (n - g0) : G;
+                if (active) {
+#pragma unroll
+                    for (int w = 0; w < G; ++w) {
+                        if (w < gw) {
+                            const int i = g0 + w;
+                            const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c);
+                            uint4 rw = make_uint4(0, 0, 0, 0);
+                            if (ROUND == INTSGD_ROUND_RANDOM)
+                                rw = philox_finish(tp, PP.tab.a[i], PP.tab.b[i], PP.tab.c[i], P.keys);
+                            uint32_t clipped = 0;
+                            consume_unit<ROUND, CLAMP>(gv, alpha2, rw, P.Lf, F01, F23, m, clipped);
+                            if (CLAMP && clipped) atomicAdd(&s_cnt[i], (u64)clipped);
+                        }
+                    }
+                }
+                mbar_arrive(&empty_bar[s]);
+            }
+            if (!ok) break;
+            if (active) {
+                int4 S;
+                if (fabsf(m) <= PP.fast_limit) {
+                    S = make_int4(__float2int_rn(F01.x), __float2int_rn(F01.y), __float2int_rn(F23.x), __float2int_rn(F23.y));
+                } else {
+                    S = redo_unit<GRAD, ROUND, CLAMP>(P, unit, alpha, step, s_cnt);
+                }
+                float4 xn;
+                xn.x = update_coord(xo.x, S.x, cdec, acc.dx2);
+                xn.y = update_coord(xo.y, S.y, cdec, acc.dx2);
+                xn.z = update_coord(xo.z, S.z, cdec, acc.dx2);
+                xn.w = update_coord(xo.w, S.w, cdec, acc.dx2);
+                store_f4<true>(P.x, unit, xn);
+                if (P.agg) store_i4<true>(P.agg, unit, S);
+                note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
+                note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
+            }
+        }
+        if (!ok) atomicExch(&s_fault, 1);
+
+        // coordinates after the last pipelined unit (at most 7): element-wise, one thread
+        if (blockIdx.x == 0 && c == 0 && ok) {
+            const int64_t j0 = PP.units << 2;
+            for (int64_t j = j0; j < P.d; ++j) {
+                int S = 0;
+                for (int i = 0; i < n; ++i) {
+                    uint32_t word = 0;
+                    if (ROUND == INTSGD_ROUND_RANDOM) {
+                        const uint4 w4 = draw_unit(j >> 2, (uint32_t)i, step, P.keys);
+                        const uint32_t wv[4] = {w4.x, w4.y, w4.z, w4.w};
+                        word = wv[j & 3];
+                    }
+                    const float y = __fmul_rn(alpha, grad_at<GRAD>(P.in[i], j));
+                    S += round_checked<ROUND>(y, word, P.Lf, &s_cnt[i], &s_cnt[INTSGD_MAX_WORKERS]);
+                }
+                apply_coord(P, j, S, cdec, acc);
+            }
+        }
+    }
+    counters_flush(s_cnt, st);   // includes a __syncthreads()
+    if (threadIdx.x == 0 && s_fault) atomicExch(&st->fault, 1);
+    grid_finalize(acc, st, P.partials, true);
+}
+
+}  // namespace intsgd

@@ -40,10 +40,11 @@ class LockStep:
     """Runs the library and the oracle side by side on full vectors."""
 
     def __init__(self, n, d, *, grad_dtype=pkg.GRAD_F32, payload_dtype=pkg.PAYLOAD_I32,
-                 rounding=pkg.ROUND_RANDOM, beta=0.9, eps=1e-8, seed=0, clip_limit=0, x0=None):
+                 rounding=pkg.ROUND_RANDOM, beta=0.9, eps=1e-8, seed=0, clip_limit=0, x0=None, fused_path=0):
         self.n, self.d = n, d
         self.lib = pkg.IntSGD(n, d, grad_dtype=grad_dtype, payload_dtype=payload_dtype, rounding=rounding,
                               beta=beta, eps=eps, seed=seed, clip_limit=clip_limit)
+        self.lib.intsgd_set_fused_path(fused_path)
         self.orc = oracle.OracleIntSGD(n, d, beta=beta, eps=eps, seed=seed, payload_dtype=payload_dtype,
                                        clip_limit=clip_limit or None, rounding=rounding)
         self.x_ref = np.ascontiguousarray(x0, dtype=np.float32).copy()

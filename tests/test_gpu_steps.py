@@ -12,11 +12,18 @@ from helpers import LockStep, check_window, dev, rel_close, to_dev, to_host
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("mode", [pkg.MODE_FUSED, pkg.MODE_TWO_KERNEL])
+FUSED_PIPELINED, FUSED_DIRECT, TWO_KERNEL = "fused-pipelined", "fused-direct", "two-kernel"
+
+
+def _mode_and_path(which):
+    return {FUSED_PIPELINED: (pkg.MODE_FUSED, 0), FUSED_DIRECT: (pkg.MODE_FUSED, 1), TWO_KERNEL: (pkg.MODE_TWO_KERNEL, 0)}[which]
+
+
+@pytest.mark.parametrize("which", [FUSED_PIPELINED, FUSED_DIRECT, TWO_KERNEL])
 @pytest.mark.parametrize("grad_dtype,payload_dtype", [(pkg.GRAD_F32, pkg.PAYLOAD_I32), (pkg.GRAD_F32, pkg.PAYLOAD_I8),
                                                       (pkg.GRAD_BF16, pkg.PAYLOAD_I8), (pkg.GRAD_BF16, pkg.PAYLOAD_I32)])
 @pytest.mark.parametrize("rounding", [pkg.ROUND_RANDOM, pkg.ROUND_NEAREST])
-def test_multi_step_lockstep(mode, grad_dtype, payload_dtype, rounding):
+def test_multi_step_lockstep(which, grad_dtype, payload_dtype, rounding):
     """Several tiles and a ragged tail: d = 5 * 2^16 + 3 spans many blocks and leaves 3 coordinates."""
     n, d, eta = 6, 5 * (1 << 16) + 3, 0.1
     rng = np.random.default_rng(21)
@@ -26,8 +33,9 @@ def test_multi_step_lockstep(mode, grad_dtype, payload_dtype, rounding):
         out[2][rng.integers(0, d, 50)] *= 300.0     # a few outliers: exercises clipping on the int8 wire
         return [synth.to_bf16_bits(g) for g in out] if grad_dtype == pkg.GRAD_BF16 else out
 
+    mode, path = _mode_and_path(which)
     ls = LockStep(n, d, grad_dtype=grad_dtype, payload_dtype=payload_dtype, rounding=rounding, seed=99,
-                  x0=rng.normal(0, 1, d).astype(np.float32))
+                  x0=rng.normal(0, 1, d).astype(np.float32), fused_path=path)
     try:
         ls.exact(grads(), eta)
         clipped = 0
@@ -58,11 +66,47 @@ def test_two_kernel_payloads_match_the_oracle():
             ls.close()
 
 
-@pytest.mark.parametrize("n,d", [(1, 1), (1, 5), (2, 3), (64, 1000), (3, 4), (16, 2)])
+@pytest.mark.parametrize("which", [FUSED_PIPELINED, FUSED_DIRECT, TWO_KERNEL])
+@pytest.mark.parametrize("grad_dtype,payload_dtype,rounding", [
+    (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM), (pkg.GRAD_BF16, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM),
+    (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_NEAREST), (pkg.GRAD_BF16, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM)])
+def test_values_outside_the_fast_range_clip_and_count_exactly(which, grad_dtype, payload_dtype, rounding):
+    """Huge, infinite and NaN gradients, and values between the fast-path range and the clip limit."""
+    n, d, eta, seed = 5, 3 * 4096 + 9, 0.1, 77
+    rng = np.random.default_rng(42)
+    mode, path = _mode_and_path(which)
+    x0 = rng.normal(0, 1, d).astype(np.float32)
+    ls = LockStep(n, d, grad_dtype=grad_dtype, payload_dtype=payload_dtype, rounding=rounding, seed=seed, x0=x0,
+                  fused_path=path)
+
+    def grads(plant):
+        out = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
+        if plant:
+            for i in range(n):
+                idx = rng.integers(0, d, 40)
+                out[i][idx[:8]] = [1e30, -1e30, np.inf, -np.inf, np.nan, 3e38, -3e38, 1e-40]
+                out[i][idx[8:24]] *= 1e4       # far outside an int8 limit, inside the int32 one
+                out[i][idx[24:]] = rng.choice([-1.0, 1.0], 16) * 10.0 ** rng.uniform(2, 7, 16)   # up to 2^27-ish
+            out[0][d - 1], out[1][d - 2], out[2][d - 9] = np.nan, np.inf, -1e25    # in the ragged tail too
+        return [synth.to_bf16_bits(g) for g in out] if grad_dtype == pkg.GRAD_BF16 else out
+
+    try:
+        ls.exact(grads(False), eta)
+        total_clip = total_nonf = 0
+        for k in range(4):
+            st, ref = ls.step(grads(True), eta, mode=mode)
+            total_clip += sum(st["clip_count"])
+            total_nonf += st["nonfinite"]
+        assert total_clip > 0 and total_nonf > 0
+    finally:
+        ls.close()
+
+
+@pytest.mark.parametrize("n,d", [(1, 1), (1, 5), (2, 3), (64, 1000), (3, 4), (16, 2), (2, 8), (3, 9), (5, 2049)])
 def test_degenerate_shapes(n, d):
     rng = np.random.default_rng(n * 1000 + d)
-    for mode in (pkg.MODE_FUSED, pkg.MODE_TWO_KERNEL):
-        ls = LockStep(n, d, seed=1, x0=rng.normal(0, 1, d).astype(np.float32))
+    for mode, path in ((pkg.MODE_FUSED, 0), (pkg.MODE_FUSED, 1), (pkg.MODE_TWO_KERNEL, 0)):
+        ls = LockStep(n, d, seed=1, x0=rng.normal(0, 1, d).astype(np.float32), fused_path=path)
         try:
             ls.exact([rng.normal(0, 1, d).astype(np.float32) for _ in range(n)], 0.1)
             for _ in range(3):
