@@ -17,7 +17,8 @@ struct intsgd_ctx {
     float Lf;             // largest fp32 <= L
     PhiloxKeys keys;
     PhiloxWorkerTable tab;
-    int fused_path;       // 0 = automatic, 1 = direct (register) kernel, 2 = pipelined kernel
+    int fused_path;       // 0 = automatic, 1 = direct (register) kernel, 2.. = pipelined kernel
+    int pipe_variant;     // index into kPipeShapes
     DevState* d_state;
     double* d_partials;
     int max_grid;
@@ -96,9 +97,7 @@ PhiloxWorkerTable make_worker_table(const PhiloxKeys& k) {
         const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)i;
         const uint32_t n0 = (uint32_t)(p1 >> 32) ^ k.k0[0];
         const uint64_t q0 = (uint64_t)0xD2511F53u * (uint64_t)n0;
-        t.a[i] = (uint32_t)p1 ^ k.k0[1];
-        t.b[i] = (uint32_t)(q0 >> 32) ^ k.k1[1];
-        t.c[i] = (uint32_t)q0;
+        t.e[i] = make_uint4((uint32_t)p1 ^ k.k0[1], (uint32_t)(q0 >> 32) ^ k.k1[1], (uint32_t)q0, 0u);
     }
     return t;
 }
@@ -205,23 +204,45 @@ void launch_fused_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStr
         fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
 
-// Pipelined kernel: kPipeConsumers consumer threads + one producer warp, kPipeGroup worker tiles per
-// stage, kPipeStages stages (192 KiB of shared memory for fp32 gradients), one block per SM.
-constexpr int kPipeConsumers = 512, kPipeGroup = 4, kPipeStages = 6;
+// Pipelined kernel shapes: NC consumer threads (+ one producer warp), UPT units per thread and
+// tile, G worker tiles per stage, NS stages; one block per SM, <= 192 KiB of shared memory.
+struct PipeShape { int nc, upt, g, ns; };
+constexpr PipeShape kPipeShapes[] = {
+    {512, 2, 4, 3},   // variant 0 (path 0 and 2): the default
+    {512, 1, 4, 6},   // variant 1
+    {512, 2, 2, 6},   // variant 2
+    {768, 1, 4, 4},   // variant 3
+    {960, 1, 2, 6},   // variant 4
+    {256, 2, 4, 6},   // variant 5
+};
+constexpr int kNumPipeShapes = sizeof(kPipeShapes) / sizeof(kPipeShapes[0]);
 
-template <int GRAD, int ROUND, bool CLAMP>
-cudaError_t launch_pipe_t(const intsgd_ctx* ctx, const PipeParams& PP, cudaStream_t s) {
-    auto kernel = fused_pipe_kernel<GRAD, ROUND, CLAMP, kPipeConsumers, kPipeGroup, kPipeStages, 1>;
+template <int GRAD, int ROUND, bool CLAMP, int V>
+cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
+    constexpr PipeShape S = kPipeShapes[V];
+    auto kernel = fused_pipe_kernel<GRAD, ROUND, CLAMP, S.nc, S.upt, S.g, S.ns>;
     const int unit_bytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
-    const int smem = kPipeStages * kPipeGroup * kPipeConsumers * unit_bytes;
+    const int smem = S.ns * S.g * S.nc * S.upt * unit_bytes;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
+    PP.tiles = (PP.units + S.nc * S.upt - 1) / (S.nc * S.upt);
     int64_t grid = PP.tiles < ctx->sm_count ? PP.tiles : ctx->sm_count;
-    kernel<<<(unsigned)grid, kPipeConsumers + 32, smem, s>>>(PP);
+    kernel<<<(unsigned)grid, S.nc + 32, smem, s>>>(PP);
     return cudaSuccess;
 }
+template <int GRAD, int ROUND, bool CLAMP>
+cudaError_t launch_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
+    switch (ctx->pipe_variant) {
+        case 1: return launch_pipe_v<GRAD, ROUND, CLAMP, 1>(ctx, PP, s);
+        case 2: return launch_pipe_v<GRAD, ROUND, CLAMP, 2>(ctx, PP, s);
+        case 3: return launch_pipe_v<GRAD, ROUND, CLAMP, 3>(ctx, PP, s);
+        case 4: return launch_pipe_v<GRAD, ROUND, CLAMP, 4>(ctx, PP, s);
+        case 5: return launch_pipe_v<GRAD, ROUND, CLAMP, 5>(ctx, PP, s);
+        default: return launch_pipe_v<GRAD, ROUND, CLAMP, 0>(ctx, PP, s);
+    }
+}
 template <int GRAD, int ROUND>
-cudaError_t launch_pipe_c(const intsgd_ctx* ctx, const PipeParams& PP, bool clamp, cudaStream_t s) {
+cudaError_t launch_pipe_c(const intsgd_ctx* ctx, PipeParams& PP, bool clamp, cudaStream_t s) {
     return clamp ? launch_pipe_t<GRAD, ROUND, true>(ctx, PP, s) : launch_pipe_t<GRAD, ROUND, false>(ctx, PP, s);
 }
 
@@ -238,7 +259,7 @@ int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     int64_t units = ctx->cfg.d >> 2;
     if (bf16) units &= ~(int64_t)1;   // bulk copies move multiples of 16 bytes
     PP.units = units;
-    PP.tiles = (units + kPipeConsumers - 1) / kPipeConsumers;
+    PP.tiles = 0;   // set by the launcher from the tile shape
     // Floors and up-decisions are summed as integer-valued floats: exact while n * (T + 1) <= 2^24.
     const float t_max = (float)((1 << 24) / ctx->cfg.n - 2);
     const bool clamp = ctx->Lf <= t_max;   // small limit (int8 wire): clamp in line, no redo for clipping
@@ -595,8 +616,10 @@ int intsgd_set_launch(intsgd_ctx* ctx, int32_t threads_per_block, int32_t blocks
 
 int intsgd_set_fused_path(intsgd_ctx* ctx, int32_t path) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
-    if (path < 0 || path > 2) return fail(ctx, INTSGD_ERR_INVALID_ARG, "path must be 0 (auto), 1 (direct) or 2 (pipelined)");
+    if (path < 0 || path >= 2 + kNumPipeShapes)
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "path must be 0 (auto), 1 (direct) or 2.. (pipelined shapes)");
     ctx->fused_path = path;
+    ctx->pipe_variant = path >= 2 ? path - 2 : 0;
     return INTSGD_OK;
 }
 

@@ -63,25 +63,36 @@ __device__ __forceinline__ float absmax_nan(float a, float b) {
     return d;
 }
 
+// 1.0f if a < b else 0.0f, in one instruction.
+__device__ __forceinline__ float lt_as_float(float a, float b) {
+    float d;
+    asm("set.lt.f32.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
 // ---- per-unit arithmetic ------------------------------------------------------------------------
 // Fast path of one worker's unit.  Floors and up-decisions are accumulated as integer-valued
 // floats (exact: the host caps the fast-path magnitude T so that n * (T + 1) <= 2^24); `m` tracks
 // max |alpha g| (NaN-propagating) so that anything outside the fast path is redone exactly.
+struct UnitAcc {
+    float2 F01, F23;   // running sums of the four coordinates
+    float m;           // running max |alpha g| over all workers (sign meaningless)
+};
+
 template <int ROUND, bool CLAMP>
-__device__ __forceinline__ void consume_unit(float4 g, float2 alpha2, uint4 w, float Lf, float2& F01, float2& F23,
-                                             float& m, uint32_t& clipped) {
+__device__ __forceinline__ void consume_unit(float4 g, float2 alpha2, uint4 w, float Lf, UnitAcc& u, uint32_t& clipped) {
     float2 y01 = __fmul2_rn(alpha2, make_float2(g.x, g.y));
     float2 y23 = __fmul2_rn(alpha2, make_float2(g.z, g.w));
-    m = absmax_nan(m, y01.x); m = absmax_nan(m, y01.y);
-    m = absmax_nan(m, y23.x); m = absmax_nan(m, y23.y);
+    u.m = absmax_nan(u.m, y01.x); u.m = absmax_nan(u.m, y01.y);
+    u.m = absmax_nan(u.m, y23.x); u.m = absmax_nan(u.m, y23.y);
     if (CLAMP) {
         clipped += (fabsf(y01.x) > Lf) + (fabsf(y01.y) > Lf) + (fabsf(y23.x) > Lf) + (fabsf(y23.y) > Lf);
         y01.x = fminf(fmaxf(y01.x, -Lf), Lf); y01.y = fminf(fmaxf(y01.y, -Lf), Lf);
         y23.x = fminf(fmaxf(y23.x, -Lf), Lf); y23.y = fminf(fmaxf(y23.y, -Lf), Lf);
     }
     if (ROUND == INTSGD_ROUND_NEAREST) {
-        F01 = __fadd2_rn(F01, make_float2(rintf(y01.x), rintf(y01.y)));
-        F23 = __fadd2_rn(F23, make_float2(rintf(y23.x), rintf(y23.y)));
+        u.F01 = __fadd2_rn(u.F01, make_float2(rintf(y01.x), rintf(y01.y)));
+        u.F23 = __fadd2_rn(u.F23, make_float2(rintf(y23.x), rintf(y23.y)));
         return;
     }
     const float2 f01 = make_float2(floorf(y01.x), floorf(y01.y));
@@ -89,12 +100,12 @@ __device__ __forceinline__ void consume_unit(float4 g, float2 alpha2, uint4 w, f
     const float2 neg1 = make_float2(-1.0f, -1.0f), scale = make_float2(16777216.0f, 16777216.0f);
     const float2 p01 = __fmul2_rn(__ffma2_rn(f01, neg1, y01), scale);   // fl32(y - f) * 2^24, both exact steps
     const float2 p23 = __fmul2_rn(__ffma2_rn(f23, neg1, y23), scale);
-    const float2 u01 = make_float2(__uint2float_rn(w.x >> 8) < p01.x ? 1.0f : 0.0f,
-                                   __uint2float_rn(w.y >> 8) < p01.y ? 1.0f : 0.0f);
-    const float2 u23 = make_float2(__uint2float_rn(w.z >> 8) < p23.x ? 1.0f : 0.0f,
-                                   __uint2float_rn(w.w >> 8) < p23.y ? 1.0f : 0.0f);
-    F01 = __fadd2_rn(__fadd2_rn(F01, f01), u01);
-    F23 = __fadd2_rn(__fadd2_rn(F23, f23), u23);
+    const float2 u01 = make_float2(lt_as_float(__uint2float_rn(w.x >> 8), p01.x),
+                                   lt_as_float(__uint2float_rn(w.y >> 8), p01.y));
+    const float2 u23 = make_float2(lt_as_float(__uint2float_rn(w.z >> 8), p23.x),
+                                   lt_as_float(__uint2float_rn(w.w >> 8), p23.y));
+    u.F01 = __fadd2_rn(__fadd2_rn(u.F01, f01), u01);
+    u.F23 = __fadd2_rn(__fadd2_rn(u.F23, f23), u23);
 }
 
 // Exact redo of one unit from global memory (rare: a value outside the fast-path range, or a
@@ -122,11 +133,10 @@ __device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float a
 }
 
 // Round-1/round-2 Philox values that depend only on (seed, worker) when the high counter word is
-// zero (d <= 2^34): computed on the host once per context.
+// zero (d <= 2^34): computed on the host once per context, copied to shared memory by each block.
+// Entry i: x = lo(M1 * i) ^ k0[1];  y = hi(M0 * n0) ^ k1[1] with n0 = hi(M1 * i) ^ k0[0];  z = lo(M0 * n0).
 struct PhiloxWorkerTable {
-    uint32_t a[INTSGD_MAX_WORKERS];   // lo(M1 * i) ^ k0[1]
-    uint32_t b[INTSGD_MAX_WORKERS];   // hi(M0 * n0) ^ k1[1],  n0 = hi(M1 * i) ^ k0[0]
-    uint32_t c[INTSGD_MAX_WORKERS];   // lo(M0 * n0)
+    uint4 e[INTSGD_MAX_WORKERS];
 };
 
 struct PipeParams {
@@ -139,7 +149,7 @@ struct PipeParams {
 
 // Philox4x32-10 for counter (unit, 0, worker, step) with rounds 1-2 folded:
 // per tile and thread: p0 = M0 * unit -> n3 = lo, n2 = hi ^ step ^ k1[0]; p1' = M1 * n2 -> H, m1.
-// per worker: m0 = H ^ a[i], m2 = b[i] ^ n3, m3 = c[i]; then rounds 3..10.
+// per worker: m0 = H ^ e[i].x, m2 = e[i].y ^ n3, m3 = e[i].z; then rounds 3..10.
 struct PhiloxThreadPart {
     uint32_t n3, H, m1;
 };
@@ -153,9 +163,8 @@ __device__ __forceinline__ PhiloxThreadPart philox_thread_part(uint32_t unit_lo,
     t.m1 = (uint32_t)p1;
     return t;
 }
-__device__ __forceinline__ uint4 philox_finish(const PhiloxThreadPart& t, uint32_t a, uint32_t b, uint32_t c,
-                                               const PhiloxKeys& K) {
-    uint32_t c0 = t.H ^ a, c1 = t.m1, c2 = b ^ t.n3, c3 = c;
+__device__ __forceinline__ uint4 philox_finish(const PhiloxThreadPart& t, uint4 e, const PhiloxKeys& K) {
+    uint32_t c0 = t.H ^ e.x, c1 = t.m1, c2 = e.y ^ t.n3, c3 = e.z;
 #pragma unroll
     for (int r = 2; r < 10; ++r) {
         const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
@@ -179,12 +188,15 @@ __device__ __forceinline__ float4 lds_unit(const unsigned char* tile, int c) {
 }
 
 // ---- the kernel ----------------------------------------------------------------------------------
-// NC consumer threads + one producer warp.  G worker tiles per stage, NS stages.
-template <int GRAD, int ROUND, bool CLAMP, int NC, int G, int NS, int MINB>
-__global__ void __launch_bounds__(NC + 32, MINB) fused_pipe_kernel(const __grid_constant__ PipeParams PP) {
+// NC consumer threads + one producer warp.  A tile is NC * UPT units; consumer c owns units
+// c, c + NC, ... of the tile.  G worker tiles per stage, NS stages.
+template <int GRAD, int ROUND, bool CLAMP, int NC, int UPT, int G, int NS>
+__global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_constant__ PipeParams PP) {
     constexpr int kUnitBytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
-    constexpr int kTileBytes = NC * kUnitBytes;
+    constexpr int kTileUnits = NC * UPT;
+    constexpr int kTileBytes = kTileUnits * kUnitBytes;
     extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(16) uint4 s_tab[INTSGD_MAX_WORKERS];
     __shared__ uint64_t full_bar[NS], empty_bar[NS];
     __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
     __shared__ int s_fault;
@@ -200,6 +212,7 @@ __global__ void __launch_bounds__(NC + 32, MINB) fused_pipe_kernel(const __grid_
         s_fault = 0;
         mbar_fence_init();
     }
+    for (int i = threadIdx.x; i < INTSGD_MAX_WORKERS; i += blockDim.x) s_tab[i] = PP.tab.e[i];
     counters_init(s_cnt);   // includes a __syncthreads()
 
     const int n = P.n;
@@ -212,8 +225,8 @@ __global__ void __launch_bounds__(NC + 32, MINB) fused_pipe_kernel(const __grid_
         if (threadIdx.x == NC) {
             uint32_t it = 0;
             for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-                const int64_t left = PP.units - tile * NC;
-                const uint32_t bytes = (uint32_t)(left < NC ? left : NC) * kUnitBytes;
+                const int64_t left = PP.units - tile * kTileUnits;
+                const uint32_t bytes = (uint32_t)(left < kTileUnits ? left : kTileUnits) * kUnitBytes;
                 const size_t offset = (size_t)tile * kTileBytes;
                 for (int g0 = 0; g0 < n; g0 += G, ++it) {
                     const uint32_t s = it % NS;
@@ -243,49 +256,77 @@ __global__ void __launch_bounds__(NC + 32, MINB) fused_pipe_kernel(const __grid_
         const float2 alpha2 = make_float2(alpha, alpha);
         uint32_t it = 0;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-            const int64_t unit = tile * NC + c;
-            const bool active = unit < PP.units;
-            float4 xo = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (active) xo = load_f4<true>(P.x, unit);
-            PhiloxThreadPart tp = {0, 0, 0};
-            if (ROUND == INTSGD_ROUND_RANDOM) tp = philox_thread_part((uint32_t)unit, step, P.keys);
-            float2 F01 = make_float2(0.f, 0.f), F23 = F01;
-            float m = 0.0f;
+            const int64_t unit0 = tile * kTileUnits + c;
+            float4 xo[UPT];
+            PhiloxThreadPart tp[UPT];
+            UnitAcc ua[UPT];
+            bool active[UPT];
+#pragma unroll
+            for (int k = 0; k < UPT; ++k) {
+                const int64_t unit = unit0 + (int64_t)k * NC;
+                active[k] = unit < PP.units;
+                xo[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (active[k]) xo[k] = load_f4<true>(P.x, unit);
+                tp[k].n3 = tp[k].H = tp[k].m1 = 0;
+                if (ROUND == INTSGD_ROUND_RANDOM) tp[k] = philox_thread_part((uint32_t)unit, step, P.keys);
+                ua[k].F01 = make_float2(0.f, 0.f);
+                ua[k].F23 = make_float2(0.f, 0.f);
+                ua[k].m = 0.0f;
+            }
             for (int g0 = 0; g0 < n; g0 += G, ++it) {
                 const uint32_t s = it % NS;
                 if (!mbar_wait(&full_bar[s], (it / NS) & 1u)) { ok = false; break; }
                 const unsigned char* src = smem + (size_t)s * G * kTileBytes;
                 const int gw = (n - g0 < G) ? (n - g0) : G;
-                if (active) {
+                if (active[UPT - 1] && gw == G) {
+                    // every unit of this thread is inside the vector and the group is full: no checks
 #pragma unroll
                     for (int w = 0; w < G; ++w) {
-                        if (w < gw) {
-                            const int i = g0 + w;
-                            const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c);
+                        const uint4 e = s_tab[g0 + w];
+#pragma unroll
+                        for (int k = 0; k < UPT; ++k) {
+                            const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
                             uint4 rw = make_uint4(0, 0, 0, 0);
-                            if (ROUND == INTSGD_ROUND_RANDOM)
-                                rw = philox_finish(tp, PP.tab.a[i], PP.tab.b[i], PP.tab.c[i], P.keys);
+                            if (ROUND == INTSGD_ROUND_RANDOM) rw = philox_finish(tp[k], e, P.keys);
                             uint32_t clipped = 0;
-                            consume_unit<ROUND, CLAMP>(gv, alpha2, rw, P.Lf, F01, F23, m, clipped);
-                            if (CLAMP && clipped) atomicAdd(&s_cnt[i], (u64)clipped);
+                            consume_unit<ROUND, CLAMP>(gv, alpha2, rw, P.Lf, ua[k], clipped);
+                            if (CLAMP && clipped) atomicAdd(&s_cnt[g0 + w], (u64)clipped);
+                        }
+                    }
+                } else {
+                    for (int w = 0; w < gw; ++w) {
+                        const uint4 e = s_tab[g0 + w];
+#pragma unroll
+                        for (int k = 0; k < UPT; ++k) {
+                            if (!active[k]) continue;
+                            const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
+                            uint4 rw = make_uint4(0, 0, 0, 0);
+                            if (ROUND == INTSGD_ROUND_RANDOM) rw = philox_finish(tp[k], e, P.keys);
+                            uint32_t clipped = 0;
+                            consume_unit<ROUND, CLAMP>(gv, alpha2, rw, P.Lf, ua[k], clipped);
+                            if (CLAMP && clipped) atomicAdd(&s_cnt[g0 + w], (u64)clipped);
                         }
                     }
                 }
                 mbar_arrive(&empty_bar[s]);
             }
             if (!ok) break;
-            if (active) {
+#pragma unroll
+            for (int k = 0; k < UPT; ++k) {
+                if (!active[k]) continue;
+                const int64_t unit = unit0 + (int64_t)k * NC;
                 int4 S;
-                if (fabsf(m) <= PP.fast_limit) {
-                    S = make_int4(__float2int_rn(F01.x), __float2int_rn(F01.y), __float2int_rn(F23.x), __float2int_rn(F23.y));
+                if (fabsf(ua[k].m) <= PP.fast_limit) {
+                    S = make_int4(__float2int_rn(ua[k].F01.x), __float2int_rn(ua[k].F01.y),
+                                  __float2int_rn(ua[k].F23.x), __float2int_rn(ua[k].F23.y));
                 } else {
                     S = redo_unit<GRAD, ROUND, CLAMP>(P, unit, alpha, step, s_cnt);
                 }
                 float4 xn;
-                xn.x = update_coord(xo.x, S.x, cdec, acc.dx2);
-                xn.y = update_coord(xo.y, S.y, cdec, acc.dx2);
-                xn.z = update_coord(xo.z, S.z, cdec, acc.dx2);
-                xn.w = update_coord(xo.w, S.w, cdec, acc.dx2);
+                xn.x = update_coord(xo[k].x, S.x, cdec, acc.dx2);
+                xn.y = update_coord(xo[k].y, S.y, cdec, acc.dx2);
+                xn.z = update_coord(xo[k].z, S.z, cdec, acc.dx2);
+                xn.w = update_coord(xo[k].w, S.w, cdec, acc.dx2);
                 store_f4<true>(P.x, unit, xn);
                 if (P.agg) store_i4<true>(P.agg, unit, S);
                 note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
