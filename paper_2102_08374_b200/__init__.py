@@ -9,4 +9,4 @@ from .binding import (  # noqa: F401
     GRAD_F32, MAX_WORKERS, MODE_EXACT, MODE_FUSED, MODE_TWO_KERNEL, OK, PAYLOAD_I8, PAYLOAD_I32,
     ROUND_NEAREST, ROUND_RANDOM, IntSGD, IntSGDError, library_path, load,
 )
-from .build import build  # noqa: F401
+from .buildlib import build  # noqa: F401

@@ -10,7 +10,7 @@ import ctypes as C
 import math
 from pathlib import Path
 
-from . import build as _build
+from . import buildlib as _build
 
 MAX_WORKERS = 64
 

@@ -217,10 +217,10 @@ constexpr PipeShape kPipeShapes[] = {
 };
 constexpr int kNumPipeShapes = sizeof(kPipeShapes) / sizeof(kPipeShapes[0]);
 
-template <int GRAD, int ROUND, bool CLAMP, int V>
+template <int GRAD, int ROUND, int V>
 cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
     constexpr PipeShape S = kPipeShapes[V];
-    auto kernel = fused_pipe_kernel<GRAD, ROUND, CLAMP, S.nc, S.upt, S.g, S.ns>;
+    auto kernel = fused_pipe_kernel<GRAD, ROUND, S.nc, S.upt, S.g, S.ns>;
     const int unit_bytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
     const int smem = S.ns * S.g * S.nc * S.upt * unit_bytes;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -230,22 +230,17 @@ cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s)
     kernel<<<(unsigned)grid, S.nc + 32, smem, s>>>(PP);
     return cudaSuccess;
 }
-template <int GRAD, int ROUND, bool CLAMP>
+template <int GRAD, int ROUND>
 cudaError_t launch_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
     switch (ctx->pipe_variant) {
-        case 1: return launch_pipe_v<GRAD, ROUND, CLAMP, 1>(ctx, PP, s);
-        case 2: return launch_pipe_v<GRAD, ROUND, CLAMP, 2>(ctx, PP, s);
-        case 3: return launch_pipe_v<GRAD, ROUND, CLAMP, 3>(ctx, PP, s);
-        case 4: return launch_pipe_v<GRAD, ROUND, CLAMP, 4>(ctx, PP, s);
-        case 5: return launch_pipe_v<GRAD, ROUND, CLAMP, 5>(ctx, PP, s);
-        default: return launch_pipe_v<GRAD, ROUND, CLAMP, 0>(ctx, PP, s);
+        case 1: return launch_pipe_v<GRAD, ROUND, 1>(ctx, PP, s);
+        case 2: return launch_pipe_v<GRAD, ROUND, 2>(ctx, PP, s);
+        case 3: return launch_pipe_v<GRAD, ROUND, 3>(ctx, PP, s);
+        case 4: return launch_pipe_v<GRAD, ROUND, 4>(ctx, PP, s);
+        case 5: return launch_pipe_v<GRAD, ROUND, 5>(ctx, PP, s);
+        default: return launch_pipe_v<GRAD, ROUND, 0>(ctx, PP, s);
     }
 }
-template <int GRAD, int ROUND>
-cudaError_t launch_pipe_c(const intsgd_ctx* ctx, PipeParams& PP, bool clamp, cudaStream_t s) {
-    return clamp ? launch_pipe_t<GRAD, ROUND, true>(ctx, PP, s) : launch_pipe_t<GRAD, ROUND, false>(ctx, PP, s);
-}
-
 bool pipe_eligible(const intsgd_ctx* ctx, bool aligned) {
     const int64_t units = ctx->cfg.d >> 2;
     return aligned && ctx->cfg.d <= ((int64_t)1 << 34) && units >= 2;
@@ -262,14 +257,13 @@ int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     PP.tiles = 0;   // set by the launcher from the tile shape
     // Floors and up-decisions are summed as integer-valued floats: exact while n * (T + 1) <= 2^24.
     const float t_max = (float)((1 << 24) / ctx->cfg.n - 2);
-    const bool clamp = ctx->Lf <= t_max;   // small limit (int8 wire): clamp in line, no redo for clipping
-    PP.fast_limit = clamp ? 3.402823466e+38f : t_max;
+    PP.fast_limit = ctx->Lf < t_max ? ctx->Lf : t_max;
     const bool nearest = ctx->cfg.rounding == INTSGD_ROUND_NEAREST;
     cudaError_t e;
-    if (!bf16 && !nearest) e = launch_pipe_c<INTSGD_GRAD_F32, INTSGD_ROUND_RANDOM>(ctx, PP, clamp, s);
-    else if (!bf16) e = launch_pipe_c<INTSGD_GRAD_F32, INTSGD_ROUND_NEAREST>(ctx, PP, clamp, s);
-    else if (!nearest) e = launch_pipe_c<INTSGD_GRAD_BF16, INTSGD_ROUND_RANDOM>(ctx, PP, clamp, s);
-    else e = launch_pipe_c<INTSGD_GRAD_BF16, INTSGD_ROUND_NEAREST>(ctx, PP, clamp, s);
+    if (!bf16 && !nearest) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_RANDOM>(ctx, PP, s);
+    else if (!bf16) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_NEAREST>(ctx, PP, s);
+    else if (!nearest) e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_RANDOM>(ctx, PP, s);
+    else e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_NEAREST>(ctx, PP, s);
     if (e != cudaSuccess) {
         std::snprintf(ctx->err, 256, "fused_pipe_kernel setup failed: %s", cudaGetErrorString(e));
         return INTSGD_ERR_CUDA;

@@ -56,10 +56,10 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
                  : "memory");
 }
 
-// max(|a|, |b|) up to sign, NaN if either is NaN.
-__device__ __forceinline__ float absmax_nan(float a, float b) {
+// max(|a|, |b|, |c|), NaN if any input is NaN (three-input max of sm_100).
+__device__ __forceinline__ float absmax3_nan(float a, float b, float c) {
     float d;
-    asm("max.NaN.xorsign.abs.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    asm("max.NaN.abs.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
 
@@ -72,24 +72,20 @@ __device__ __forceinline__ float lt_as_float(float a, float b) {
 
 // ---- per-unit arithmetic ------------------------------------------------------------------------
 // Fast path of one worker's unit.  Floors and up-decisions are accumulated as integer-valued
-// floats (exact: the host caps the fast-path magnitude T so that n * (T + 1) <= 2^24); `m` tracks
-// max |alpha g| (NaN-propagating) so that anything outside the fast path is redone exactly.
+// floats (exact: the host caps the fast-path magnitude T so that n * (T + 1) <= 2^24, and T never
+// exceeds the clip limit); `m` tracks max |alpha g| (NaN-propagating) so that a unit with any value
+// outside the fast range -- clipped, huge or not finite -- is redone exactly at the end of its tile.
 struct UnitAcc {
     float2 F01, F23;   // running sums of the four coordinates
-    float m;           // running max |alpha g| over all workers (sign meaningless)
+    float m;           // running max |alpha g| over all workers
 };
 
-template <int ROUND, bool CLAMP>
-__device__ __forceinline__ void consume_unit(float4 g, float2 alpha2, uint4 w, float Lf, UnitAcc& u, uint32_t& clipped) {
-    float2 y01 = __fmul2_rn(alpha2, make_float2(g.x, g.y));
-    float2 y23 = __fmul2_rn(alpha2, make_float2(g.z, g.w));
-    u.m = absmax_nan(u.m, y01.x); u.m = absmax_nan(u.m, y01.y);
-    u.m = absmax_nan(u.m, y23.x); u.m = absmax_nan(u.m, y23.y);
-    if (CLAMP) {
-        clipped += (fabsf(y01.x) > Lf) + (fabsf(y01.y) > Lf) + (fabsf(y23.x) > Lf) + (fabsf(y23.y) > Lf);
-        y01.x = fminf(fmaxf(y01.x, -Lf), Lf); y01.y = fminf(fmaxf(y01.y, -Lf), Lf);
-        y23.x = fminf(fmaxf(y23.x, -Lf), Lf); y23.y = fminf(fmaxf(y23.y, -Lf), Lf);
-    }
+template <int ROUND>
+__device__ __forceinline__ void consume_unit(float4 g, float2 alpha2, uint4 w, UnitAcc& u) {
+    const float2 y01 = __fmul2_rn(alpha2, make_float2(g.x, g.y));
+    const float2 y23 = __fmul2_rn(alpha2, make_float2(g.z, g.w));
+    u.m = absmax3_nan(u.m, y01.x, y01.y);
+    u.m = absmax3_nan(u.m, y23.x, y23.y);
     if (ROUND == INTSGD_ROUND_NEAREST) {
         u.F01 = __fadd2_rn(u.F01, make_float2(rintf(y01.x), rintf(y01.y)));
         u.F23 = __fadd2_rn(u.F23, make_float2(rintf(y23.x), rintf(y23.y)));
@@ -108,9 +104,9 @@ __device__ __forceinline__ void consume_unit(float4 g, float2 alpha2, uint4 w, f
     u.F23 = __fadd2_rn(__fadd2_rn(u.F23, f23), u23);
 }
 
-// Exact redo of one unit from global memory (rare: a value outside the fast-path range, or a
-// NaN/Inf).  In CLAMP mode the fast path has already counted |y| > Lf, so only NaN adds a clip.
-template <int GRAD, int ROUND, bool CLAMP>
+// Exact redo of one unit from global memory with the full clipping rule and the counters (rare:
+// some |alpha g| outside the fast range, or a NaN/Inf).  The fast path has counted nothing.
+template <int GRAD, int ROUND>
 __device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float alpha, uint32_t step, u64* s_cnt) {
     int S[4] = {0, 0, 0, 0};
     for (int i = 0; i < P.n; ++i) {
@@ -121,12 +117,7 @@ __device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float a
         const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
         for (int e = 0; e < 4; ++e) {
             const float y = __fmul_rn(alpha, gv[e]);
-            const bool in = fabsf(y) <= P.Lf;
-            if (in) { S[e] += round_in_range<ROUND>(y, wv[e]); continue; }
-            const bool is_nan = (y != y);
-            if (!CLAMP || is_nan) atomicAdd(&s_cnt[i], 1ull);
-            if (!(fabsf(y) <= 3.402823466e+38f)) atomicAdd(&s_cnt[INTSGD_MAX_WORKERS], 1ull);
-            S[e] += is_nan ? 0 : (y > 0.0f ? (int)P.Lf : -(int)P.Lf);
+            S[e] += round_checked<ROUND>(y, wv[e], P.Lf, &s_cnt[i], &s_cnt[INTSGD_MAX_WORKERS]);
         }
     }
     return make_int4(S[0], S[1], S[2], S[3]);
@@ -190,7 +181,7 @@ __device__ __forceinline__ float4 lds_unit(const unsigned char* tile, int c) {
 // ---- the kernel ----------------------------------------------------------------------------------
 // NC consumer threads + one producer warp.  A tile is NC * UPT units; consumer c owns units
 // c, c + NC, ... of the tile.  G worker tiles per stage, NS stages.
-template <int GRAD, int ROUND, bool CLAMP, int NC, int UPT, int G, int NS>
+template <int GRAD, int ROUND, int NC, int UPT, int G, int NS>
 __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_constant__ PipeParams PP) {
     constexpr int kUnitBytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
     constexpr int kTileUnits = NC * UPT;
@@ -223,19 +214,20 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
     if (threadIdx.x >= NC) {
         // ------------------------------- producer ---------------------------------------------
         if (threadIdx.x == NC) {
-            uint32_t it = 0;
+            uint32_t it = 0, s = 0, phase = 0;   // it: stages filled so far; s = it % NS; phase = (it / NS) & 1
             for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
                 const int64_t left = PP.units - tile * kTileUnits;
                 const uint32_t bytes = (uint32_t)(left < kTileUnits ? left : kTileUnits) * kUnitBytes;
                 const size_t offset = (size_t)tile * kTileBytes;
-                for (int g0 = 0; g0 < n; g0 += G, ++it) {
-                    const uint32_t s = it % NS;
-                    if (it >= NS && !mbar_wait(&empty_bar[s], ((it / NS) & 1u) ^ 1u)) { ok = false; break; }
+                for (int g0 = 0; g0 < n; g0 += G) {
+                    if (it >= NS && !mbar_wait(&empty_bar[s], phase ^ 1u)) { ok = false; break; }
                     const int gw = (n - g0 < G) ? (n - g0) : G;
                     mbar_arrive_expect_tx(&full_bar[s], (uint32_t)gw * bytes);
                     unsigned char* dst = smem + (size_t)s * G * kTileBytes;
                     for (int w = 0; w < gw; ++w)
                         bulk_load(dst + w * kTileBytes, (const unsigned char*)P.in[g0 + w] + offset, bytes, &full_bar[s]);
+                    ++it;
+                    if (++s == NS) { s = 0; phase ^= 1u; }
                 }
             }
             if (!ok) {
@@ -254,7 +246,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         const float alpha = st->alpha, cdec = st->c;
         const uint32_t step = st->step;
         const float2 alpha2 = make_float2(alpha, alpha);
-        uint32_t it = 0;
+        uint32_t s = 0, phase = 0;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             const int64_t unit0 = tile * kTileUnits + c;
             float4 xo[UPT];
@@ -273,9 +265,8 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 ua[k].F23 = make_float2(0.f, 0.f);
                 ua[k].m = 0.0f;
             }
-            for (int g0 = 0; g0 < n; g0 += G, ++it) {
-                const uint32_t s = it % NS;
-                if (!mbar_wait(&full_bar[s], (it / NS) & 1u)) { ok = false; break; }
+            for (int g0 = 0; g0 < n; g0 += G) {
+                if (!mbar_wait(&full_bar[s], phase)) { ok = false; break; }
                 const unsigned char* src = smem + (size_t)s * G * kTileBytes;
                 const int gw = (n - g0 < G) ? (n - g0) : G;
                 if (active[UPT - 1] && gw == G) {
@@ -288,9 +279,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
                             uint4 rw = make_uint4(0, 0, 0, 0);
                             if (ROUND == INTSGD_ROUND_RANDOM) rw = philox_finish(tp[k], e, P.keys);
-                            uint32_t clipped = 0;
-                            consume_unit<ROUND, CLAMP>(gv, alpha2, rw, P.Lf, ua[k], clipped);
-                            if (CLAMP && clipped) atomicAdd(&s_cnt[g0 + w], (u64)clipped);
+                            consume_unit<ROUND>(gv, alpha2, rw, ua[k]);
                         }
                     }
                 } else {
@@ -302,13 +291,12 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
                             uint4 rw = make_uint4(0, 0, 0, 0);
                             if (ROUND == INTSGD_ROUND_RANDOM) rw = philox_finish(tp[k], e, P.keys);
-                            uint32_t clipped = 0;
-                            consume_unit<ROUND, CLAMP>(gv, alpha2, rw, P.Lf, ua[k], clipped);
-                            if (CLAMP && clipped) atomicAdd(&s_cnt[g0 + w], (u64)clipped);
+                            consume_unit<ROUND>(gv, alpha2, rw, ua[k]);
                         }
                     }
                 }
                 mbar_arrive(&empty_bar[s]);
+                if (++s == NS) { s = 0; phase ^= 1u; }
             }
             if (!ok) break;
 #pragma unroll
@@ -316,11 +304,11 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 if (!active[k]) continue;
                 const int64_t unit = unit0 + (int64_t)k * NC;
                 int4 S;
-                if (fabsf(ua[k].m) <= PP.fast_limit) {
+                if (ua[k].m <= PP.fast_limit) {
                     S = make_int4(__float2int_rn(ua[k].F01.x), __float2int_rn(ua[k].F01.y),
                                   __float2int_rn(ua[k].F23.x), __float2int_rn(ua[k].F23.y));
                 } else {
-                    S = redo_unit<GRAD, ROUND, CLAMP>(P, unit, alpha, step, s_cnt);
+                    S = redo_unit<GRAD, ROUND>(P, unit, alpha, step, s_cnt);
                 }
                 float4 xn;
                 xn.x = update_coord(xo[k].x, S.x, cdec, acc.dx2);
