@@ -47,6 +47,7 @@ extern "C" {
 #define INTSGD_ERR_CUDA             -3   /* a CUDA runtime call failed; see intsgd_last_error */
 #define INTSGD_ERR_SCALE_NONFINITE  -4   /* alpha_k or c_k not finite or not positive; step not applied */
 #define INTSGD_ERR_UNSUPPORTED      -5   /* valid request this build does not implement */
+#define INTSGD_ERR_TOO_LARGE        -7   /* intsgd_sqdiff_noalloc: d exceeds INTSGD_NOALLOC_MAX_D */
 #define INTSGD_ERR_TIMEOUT          -6   /* a bounded wait inside a kernel gave up; that step's results are
                                             invalid; sticky until intsgd_set_state */
 
@@ -172,6 +173,24 @@ int intsgd_set_fused_path(intsgd_ctx* ctx, int32_t path);
 
 /* Number of kernels this library has launched on the context since creation. */
 int64_t intsgd_launch_count(const intsgd_ctx* ctx);
+
+/* ||x - x_prev||^2 for callers that must not allocate device memory (the paper has no counterpart:
+ * this is an addition for hosts that cannot create a context, because intsgd_create calls cudaMalloc
+ * -- e.g. a process whose framework owns all device memory and forbids raw allocations, a loop that
+ * cannot afford the allocator's implicit synchronisation, or a plug-in that is handed only buffers and
+ * a stream).  Needs no context and calls no cudaMalloc / cudaFree or allocating routine: the reduction
+ * scratch is a fixed array inside the library image, 128 KiB + 8 bytes on every GPU that loads the
+ * library, held until the process exits.
+ *   x, x_prev : device, d floats each, 4-byte aligned (16-byte aligned pointers use vector loads)
+ *   out       : device, one double, 8-byte aligned; receives sum_j fl32(x_j - x_prev_j)^2 in fp64
+ *   d         : 1 .. INTSGD_NOALLOC_MAX_D; larger -> INTSGD_ERR_TOO_LARGE, nothing is enqueued
+ * Works on the current device and enqueues on `stream` without synchronising.  The first call on
+ * each device looks up the array's device address (cudaGetSymbolAddress); make that first call
+ * before any stream capture.  All calls on a device share the array: it keeps the previous call's
+ * partial sums, its arrival counter is cleared on `stream` before every launch, and two calls that
+ * overlap on the GPU race.  The summation order depends on d only. */
+#define INTSGD_NOALLOC_MAX_D ((int64_t)1 << 28)
+int intsgd_sqdiff_noalloc(const float* x, const float* x_prev, int64_t d, double* out, void* stream);
 
 /* Static, NUL-terminated description of the last failing call ("" if none); never NULL.
  * ctx may be NULL to read the message of a failed intsgd_create on this thread. */

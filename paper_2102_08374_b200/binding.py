@@ -21,6 +21,8 @@ ERR_CUDA = -3
 ERR_SCALE_NONFINITE = -4
 ERR_UNSUPPORTED = -5
 ERR_TIMEOUT = -6
+ERR_TOO_LARGE = -7
+NOALLOC_MAX_D = 1 << 28
 
 GRAD_F32, GRAD_BF16 = 0, 1
 PAYLOAD_I32, PAYLOAD_I8 = 0, 1
@@ -31,6 +33,7 @@ EXPORTS = [
     "intsgd_create", "intsgd_destroy", "intsgd_scale", "intsgd_sqdiff", "intsgd_encode",
     "intsgd_aggregate", "intsgd_step", "intsgd_step_host", "intsgd_get_stats", "intsgd_get_state",
     "intsgd_set_state", "intsgd_set_launch", "intsgd_set_fused_path", "intsgd_launch_count", "intsgd_last_error",
+    "intsgd_sqdiff_noalloc",
 ]
 
 
@@ -87,6 +90,7 @@ def load() -> C.CDLL:
     lib.intsgd_set_state.argtypes = [vp, C.POINTER(State)]
     lib.intsgd_set_launch.argtypes = [vp, i32, i32]
     lib.intsgd_set_fused_path.argtypes = [vp, i32]
+    lib.intsgd_sqdiff_noalloc.argtypes = [vp, vp, i64, vp, vp]
     lib.intsgd_launch_count.argtypes = [vp]
     lib.intsgd_launch_count.restype = i64
     lib.intsgd_last_error.argtypes = [vp]
@@ -113,6 +117,22 @@ def _addr(t) -> int | None:
 
 def _ptr_array(seq):
     return (C.c_void_p * len(seq))(*[_addr(t) for t in seq])
+
+
+def intsgd_sqdiff_noalloc(x, x_prev, d, out, stream=None) -> None:
+    """``out[0] = ||x - x_prev||^2`` on the current device without any device allocation.
+
+    For hosts that cannot create a context (``intsgd_create`` calls ``cudaMalloc``): the reduction
+    scratch is a fixed 128 KiB array inside the library.  ``x``, ``x_prev``: d floats on the device;
+    ``out``: one device double.  ``d`` may not exceed ``NOALLOC_MAX_D``.  Calls on one device share
+    the scratch, so they must not overlap on the GPU.
+    """
+    rc = load().intsgd_sqdiff_noalloc(_addr(x), _addr(x_prev), d, _addr(out), stream)
+    if rc != OK:
+        what = {ERR_TOO_LARGE: f"d = {d} exceeds the fixed scratch (max {NOALLOC_MAX_D} coordinates)",
+                ERR_INVALID_ARG: "null pointer or d < 1", ERR_ALIGN: "pointer not aligned to its element size",
+                ERR_CUDA: "a CUDA runtime call failed"}.get(rc, "failed")
+        raise IntSGDError(rc, f"intsgd_sqdiff_noalloc: {what}")
 
 
 class IntSGD:

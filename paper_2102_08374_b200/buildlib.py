@@ -9,7 +9,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libintsgd.so"
-SOURCES = [CSRC / "intsgd.cu"]
+SOURCES = [CSRC / "intsgd.cu", CSRC / "intsgd_noalloc.cu"]
 HEADERS = [CSRC / "intsgd_device.cuh", CSRC / "intsgd_kernels.cuh", CSRC / "intsgd_pipe.cuh", ROOT / "include" / "intsgd.h"]
 
 NVCC_FLAGS = [
