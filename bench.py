@@ -189,7 +189,7 @@ def main():
 
     import torch
     import paper_2102_08374_b200 as pkg
-    from paper_2102_08374_b200 import synth
+    from paper_2102_08374_b200 import replicas, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -210,7 +210,7 @@ def main():
     mode = pkg.MODE_TWO_KERNEL if args.mode == "two_kernel" else pkg.MODE_FUSED
     gb, pb = (2 if args.grad == "bf16" else 4), (1 if args.payload == "int8" else 4)
 
-    grads = synth.bucket_gradients_device(n, d, device, seed_base=500 + 1000 * rank,
+    grads = synth.bucket_gradients_device(n, d, device, seed_base=replicas.rank_seed_base(rank),
                                           dtype=torch.bfloat16 if args.grad == "bf16" else None)
     x = synth.iterate_device(d, device)
     agg = torch.empty(d, dtype=torch.int32, device=device)
@@ -256,11 +256,7 @@ def main():
     total_ms = events[0].elapsed_time(events[K])
     per_step_ms = [events[k].elapsed_time(events[k + 1]) for k in range(K)]
     st = lib.intsgd_get_stats()
-    if dist is not None:
-        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-
+    total_ms = replicas.max_over_ranks(dist, total_ms, device)
     value = world * n * d * K / (total_ms * 1e-3)
     bytes_per_launch = algorithmic_bytes_per_coordinate(n, gb, pb, args.mode) * d
     avg_ms = statistics.mean(per_step_ms)
@@ -290,10 +286,7 @@ def main():
         ev1.record()
         torch.cuda.synchronize()
         e2e_ms = ev0.elapsed_time(ev1)
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = replicas.max_over_ranks(dist, e2e_ms, device)
         e2e = {"value": world * n * d * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": n * d * gb + d * 4, "d2h_bytes_per_step": d * 8,
                "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,

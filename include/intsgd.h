@@ -167,8 +167,9 @@ int intsgd_set_launch(intsgd_ctx* ctx, int32_t threads_per_block, int32_t blocks
 
 /* Which kernel runs INTSGD_MODE_FUSED: 0 = automatic (the pipelined kernel -- bulk asynchronous copies
  * into a shared-memory ring -- when every pointer is 16-byte aligned and d <= 2^34, else the direct
- * kernel), 1 = always the direct kernel, 2 = same as 0.  Both give identical x, aggregate and
- * counters; dx2 differs only by summation order. */
+ * kernel), 1 = always the direct kernel, 2 = same as 0, 3 and 4 = the pipelined kernel with other
+ * tile shapes (kept for tuning).  All give identical x, aggregate and counters; dx2 differs only
+ * by summation order. */
 int intsgd_set_fused_path(intsgd_ctx* ctx, int32_t path);
 
 /* Number of kernels this library has launched on the context since creation. */

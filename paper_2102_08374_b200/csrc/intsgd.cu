@@ -208,12 +208,9 @@ void launch_fused_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStr
 // tile, G worker tiles per stage, NS stages; one block per SM, <= 192 KiB of shared memory.
 struct PipeShape { int nc, upt, g, ns; };
 constexpr PipeShape kPipeShapes[] = {
-    {512, 2, 4, 3},   // variant 0 (path 0 and 2): the default
-    {512, 1, 4, 6},   // variant 1
-    {512, 2, 2, 6},   // variant 2
-    {768, 1, 4, 4},   // variant 3
-    {960, 1, 2, 6},   // variant 4
-    {256, 2, 4, 6},   // variant 5
+    {512, 2, 4, 3},   // variant 0 (path 0 and 2): the default, fastest of the shapes tried on B200
+    {512, 1, 4, 6},   // variant 1 (path 3): one unit per thread, deeper ring
+    {256, 4, 4, 3},   // variant 2 (path 4): fewer, fatter threads
 };
 constexpr int kNumPipeShapes = sizeof(kPipeShapes) / sizeof(kPipeShapes[0]);
 
@@ -235,9 +232,6 @@ cudaError_t launch_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s)
     switch (ctx->pipe_variant) {
         case 1: return launch_pipe_v<GRAD, ROUND, 1>(ctx, PP, s);
         case 2: return launch_pipe_v<GRAD, ROUND, 2>(ctx, PP, s);
-        case 3: return launch_pipe_v<GRAD, ROUND, 3>(ctx, PP, s);
-        case 4: return launch_pipe_v<GRAD, ROUND, 4>(ctx, PP, s);
-        case 5: return launch_pipe_v<GRAD, ROUND, 5>(ctx, PP, s);
         default: return launch_pipe_v<GRAD, ROUND, 0>(ctx, PP, s);
     }
 }
