@@ -264,3 +264,68 @@ class OracleIntSGD:
         self.step += 1
         out.update(r=r, alpha64=a64, alpha=a32, c=c32)
         return out
+
+
+class OracleIntSGDBlocks:
+    """Algorithm 2 (adaptive block quantization): one moving average r_{k,l} and one scale
+    alpha_{k,l} = eta sqrt(d_l) / sqrt(2 n r_{k,l} + eta^2 (d_l / d) eps^2) per block l of
+    coordinates [offsets[l], offsets[l+1]).  Each block is rounded, summed, decoded and applied with
+    its own scale; the random stream is still indexed by the absolute coordinate.  Step 0 is the
+    exact first communication, as in Algorithm 1.
+    """
+
+    def __init__(self, n, offsets, *, beta=0.9, eps=1e-8, seed=0, payload_dtype=PAYLOAD_I32,
+                 clip_limit=None, rounding=ROUND_RANDOM):
+        self.offsets = [int(o) for o in offsets]
+        assert self.offsets[0] == 0 and all(a < b for a, b in zip(self.offsets, self.offsets[1:]))
+        self.n, self.d, self.B = n, self.offsets[-1], len(self.offsets) - 1
+        self.beta, self.eps, self.seed = beta, eps, seed
+        self.payload_dtype, self.rounding = payload_dtype, rounding
+        self.clip_limit = default_clip_limit(n, payload_dtype) if not clip_limit else clip_limit
+        self.r = [0.0] * self.B
+        self.dx2 = [0.0] * self.B
+        self.step = 0
+
+    def _block_dx2(self, x_new, x_old):
+        return [sqdiff(x_new[a:b], x_old[a:b]) for a, b in zip(self.offsets, self.offsets[1:])]
+
+    def exact_step(self, grads, x, eta):
+        x_old = x.copy()
+        exact_step(grads, x, eta)
+        self.dx2 = self._block_dx2(x, x_old)
+        self.step += 1
+        return dict(dx2=list(self.dx2))
+
+    def scales(self, eta, dx2=None):
+        dx2 = self.dx2 if dx2 is None else dx2
+        out = []
+        for l, (a, b) in enumerate(zip(self.offsets, self.offsets[1:])):
+            out.append(scale_block(self.d, b - a, self.n, eta, self.beta, self.eps, self.r[l], dx2[l]))
+        return out   # list of (r, alpha64, alpha32, c32)
+
+    def int_step(self, grads, x, eta, *, alpha_c=None, want_agg=True):
+        """alpha_c: optional list of (alpha32, c32) per block imposed on the vector part."""
+        sc = self.scales(eta)
+        self.r = [t[0] for t in sc]
+        agg = np.empty(self.d, dtype=np.int32) if want_agg else None
+        clip = [0] * self.n
+        nonf = ovf = mx = 0
+        new_dx2 = []
+        for l, (a, b) in enumerate(zip(self.offsets, self.offsets[1:])):
+            alpha, c = (sc[l][2], sc[l][3]) if alpha_c is None else alpha_c[l]
+            xw = x[a:b]   # a view: updated in place
+            out = step_window([g[a:b] for g in grads], xw, alpha, c, step=self.step, seed=self.seed, j0=a,
+                              clip_limit=self.clip_limit, payload_dtype=self.payload_dtype,
+                              rounding=self.rounding, want_agg=want_agg)
+            if want_agg:
+                agg[a:b] = out["agg"]
+            clip = [u + v for u, v in zip(clip, out["clip_count"])]
+            nonf += out["nonfinite"]
+            ovf += out["agg_overflow"]
+            mx = max(mx, out["max_abs_agg"])
+            new_dx2.append(out["dx2"])
+        self.dx2 = new_dx2
+        self.step += 1
+        return dict(agg=agg, dx2=list(new_dx2), r=list(self.r), alpha64=[t[1] for t in sc],
+                    alpha=[t[2] for t in sc], c=[t[3] for t in sc], clip_count=clip, nonfinite=nonf,
+                    agg_overflow=ovf, max_abs_agg=mx)
