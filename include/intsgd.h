@@ -39,6 +39,7 @@ extern "C" {
 #endif
 
 #define INTSGD_MAX_WORKERS 64
+#define INTSGD_MAX_BLOCKS  4096
 
 /* status codes */
 #define INTSGD_OK                    0
@@ -159,6 +160,23 @@ int intsgd_get_stats(intsgd_ctx* ctx, intsgd_stats* out);
 int intsgd_get_state(intsgd_ctx* ctx, intsgd_state* out);
 /* Overwrite the scalar state (checkpoint resume; tests that impose alpha and c). */
 int intsgd_set_state(intsgd_ctx* ctx, const intsgd_state* in);
+
+/* Block-wise scales (Algorithm 2, "adaptive block quantization"; Proposition 4): the coordinates are
+ * split into num_blocks contiguous blocks [offsets[l], offsets[l+1]) -- for instance one per layer --
+ * and each block keeps its own moving average and scale:
+ *     r_{k,l}     = beta r_{k-1,l} + (1 - beta) ||(x^k)_l - (x^{k-1})_l||^2
+ *     alpha_{k,l} = eta_k sqrt(d_l) / sqrt(2 n r_{k,l} + eta_k^2 (d_l / d) eps^2)
+ * offsets: HOST array of num_blocks + 1 values, offsets[0] = 0, strictly increasing, last = d.
+ * num_blocks = 0 returns to the single scalar alpha of Algorithm 1.  The call synchronises,
+ * allocates the per-block state (r = 0, dx2 = 0) and d/128 doubles of reduction scratch.
+ * With a partition set, intsgd_step supports INTSGD_MODE_EXACT and INTSGD_MODE_FUSED (intsgd_scale
+ * computes all block scales; dx2_override must be negative); intsgd_sqdiff / encode / aggregate and
+ * INTSGD_MODE_TWO_KERNEL return INTSGD_ERR_UNSUPPORTED.  intsgd_state.dx2 is the sum over blocks,
+ * .alpha and .c are those of block 0; counters are unchanged. */
+int intsgd_set_blocks(intsgd_ctx* ctx, int32_t num_blocks, const int64_t* offsets);
+/* Per-block state, HOST arrays of num_blocks values each (any may be NULL); both calls synchronise. */
+int intsgd_get_block_state(intsgd_ctx* ctx, double* r, double* dx2, float* alpha, float* c);
+int intsgd_set_block_state(intsgd_ctx* ctx, const double* r, const double* dx2);
 
 /* Tuning knob: threads per block (multiple of 32, <= 512) and resident blocks per SM used to
  * size the grids of the vector kernels.  0 keeps the built-in value.  Results do not depend on

@@ -33,7 +33,7 @@ EXPORTS = [
     "intsgd_create", "intsgd_destroy", "intsgd_scale", "intsgd_sqdiff", "intsgd_encode",
     "intsgd_aggregate", "intsgd_step", "intsgd_step_host", "intsgd_get_stats", "intsgd_get_state",
     "intsgd_set_state", "intsgd_set_launch", "intsgd_set_fused_path", "intsgd_launch_count", "intsgd_last_error",
-    "intsgd_sqdiff_noalloc",
+    "intsgd_sqdiff_noalloc", "intsgd_set_blocks", "intsgd_get_block_state", "intsgd_set_block_state",
 ]
 
 
@@ -90,6 +90,9 @@ def load() -> C.CDLL:
     lib.intsgd_set_state.argtypes = [vp, C.POINTER(State)]
     lib.intsgd_set_launch.argtypes = [vp, i32, i32]
     lib.intsgd_set_fused_path.argtypes = [vp, i32]
+    lib.intsgd_set_blocks.argtypes = [vp, i32, C.POINTER(C.c_int64)]
+    lib.intsgd_get_block_state.argtypes = [vp, vp, vp, vp, vp]
+    lib.intsgd_set_block_state.argtypes = [vp, vp, vp]
     lib.intsgd_sqdiff_noalloc.argtypes = [vp, vp, i64, vp, vp]
     lib.intsgd_launch_count.argtypes = [vp]
     lib.intsgd_launch_count.restype = i64
@@ -151,6 +154,7 @@ class IntSGD:
             self._ctx = C.c_void_p()
             raise IntSGDError(rc, msg)
         self.n, self.d = n, d
+        self.num_blocks = 0
 
     # -- lifetime ---------------------------------------------------------------------------
     def close(self):
@@ -218,6 +222,29 @@ class IntSGD:
 
     def intsgd_set_launch(self, threads_per_block=0, blocks_per_sm=0):
         self._check(self._lib.intsgd_set_launch(self._ctx, threads_per_block, blocks_per_sm))
+
+    def intsgd_set_blocks(self, offsets):
+        """Block partition for Algorithm 2; ``offsets`` has num_blocks + 1 entries (empty/None = off)."""
+        offsets = list(offsets) if offsets is not None else []
+        B = max(len(offsets) - 1, 0)
+        arr = (C.c_int64 * (B + 1))(*offsets) if B else None
+        self._check(self._lib.intsgd_set_blocks(self._ctx, B, arr))
+        self.num_blocks = B
+
+    def intsgd_get_block_state(self) -> dict:
+        B = self.num_blocks
+        r, dx2 = (C.c_double * B)(), (C.c_double * B)()
+        alpha, c = (C.c_float * B)(), (C.c_float * B)()
+        self._check(self._lib.intsgd_get_block_state(self._ctx, C.addressof(r), C.addressof(dx2),
+                                                     C.addressof(alpha), C.addressof(c)))
+        return dict(r=list(r), dx2=list(dx2), alpha=list(alpha), c=list(c))
+
+    def intsgd_set_block_state(self, r=None, dx2=None):
+        B = self.num_blocks
+        ra = (C.c_double * B)(*r) if r is not None else None
+        da = (C.c_double * B)(*dx2) if dx2 is not None else None
+        self._check(self._lib.intsgd_set_block_state(self._ctx, C.addressof(ra) if ra is not None else None,
+                                                     C.addressof(da) if da is not None else None))
 
     def intsgd_set_fused_path(self, path: int):
         self._check(self._lib.intsgd_set_fused_path(self._ctx, path))

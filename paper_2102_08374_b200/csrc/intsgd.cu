@@ -27,6 +27,9 @@ struct intsgd_ctx {
     int blocks_per_sm;
     cudaStream_t last_stream;
     int64_t launches;
+    // block-wise scales (Algorithm 2); bs.B == 0 means one scalar alpha
+    BlockState bs;
+    int64_t* d_offsets;
     // device staging for intsgd_step_host (allocated on first use)
     void* stage_grads[INTSGD_MAX_WORKERS];
     float* stage_x;
@@ -152,6 +155,13 @@ int launch_scale(intsgd_ctx* ctx, double eta, double dx2_override, cudaStream_t 
     if (std::isnan(dx2_override) || std::isinf(dx2_override))
         return fail(ctx, INTSGD_ERR_INVALID_ARG, "dx2_override must be finite (negative = use the state)");
     const double dd = (double)ctx->cfg.d, dn = (double)ctx->cfg.n;
+    if (ctx->bs.B > 0) {
+        if (dx2_override >= 0.0)
+            return fail(ctx, INTSGD_ERR_UNSUPPORTED, "dx2_override is not available with block-wise scales");
+        scale_blocks_kernel<<<1, 1024, 0, s>>>(ctx->d_state, ctx->bs, dd, 2.0 * dn, dn, eta, ctx->cfg.beta, ctx->cfg.eps,
+                                               ctx->cfg.n);
+        return after_launch(ctx, "scale_blocks_kernel");
+    }
     scale_kernel<<<1, 32, 0, s>>>(ctx->d_state, std::sqrt(dd), 2.0 * dn, dn, eta, ctx->cfg.beta, ctx->cfg.eps,
                                   dx2_override, ctx->cfg.n);
     return after_launch(ctx, "scale_kernel");
@@ -214,10 +224,10 @@ constexpr PipeShape kPipeShapes[] = {
 };
 constexpr int kNumPipeShapes = sizeof(kPipeShapes) / sizeof(kPipeShapes[0]);
 
-template <int GRAD, int ROUND, int V>
+template <int GRAD, int ROUND, bool BLOCKS, int V>
 cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
     constexpr PipeShape S = kPipeShapes[V];
-    auto kernel = fused_pipe_kernel<GRAD, ROUND, S.nc, S.upt, S.g, S.ns>;
+    auto kernel = fused_pipe_kernel<GRAD, ROUND, BLOCKS, S.nc, S.upt, S.g, S.ns>;
     const int unit_bytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
     const int smem = S.ns * S.g * S.nc * S.upt * unit_bytes;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -229,15 +239,33 @@ cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s)
 }
 template <int GRAD, int ROUND>
 cudaError_t launch_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
+    if (ctx->bs.B > 0) return launch_pipe_v<GRAD, ROUND, true, 0>(ctx, PP, s);   // block-wise: default shape only
     switch (ctx->pipe_variant) {
-        case 1: return launch_pipe_v<GRAD, ROUND, 1>(ctx, PP, s);
-        case 2: return launch_pipe_v<GRAD, ROUND, 2>(ctx, PP, s);
-        default: return launch_pipe_v<GRAD, ROUND, 0>(ctx, PP, s);
+        case 1: return launch_pipe_v<GRAD, ROUND, false, 1>(ctx, PP, s);
+        case 2: return launch_pipe_v<GRAD, ROUND, false, 2>(ctx, PP, s);
+        default: return launch_pipe_v<GRAD, ROUND, false, 0>(ctx, PP, s);
     }
 }
 bool pipe_eligible(const intsgd_ctx* ctx, bool aligned) {
     const int64_t units = ctx->cfg.d >> 2;
     return aligned && ctx->cfg.d <= ((int64_t)1 << 34) && units >= 2;
+}
+
+void fill_block_params(const intsgd_ctx* ctx, VecParams& P, int64_t covered_end) {
+    P.bp.offsets = ctx->bs.offsets;
+    P.bp.alpha = ctx->bs.alpha;
+    P.bp.c = ctx->bs.c;
+    P.bp.chunk_sum = ctx->bs.chunk_sum;
+    P.bp.edge_sum = ctx->bs.edge_sum;
+    P.bp.tail_sq = ctx->bs.tail_sq;
+    P.bp.covered_end = covered_end;
+    P.bp.B = ctx->bs.B;
+}
+
+// Finishes a block-wise step: per-segment squared step lengths, total, step counter.
+int launch_block_norm(intsgd_ctx* ctx, int64_t covered_end, bool check_status, cudaStream_t s) {
+    block_norm_kernel<<<ctx->bs.B, 256, 0, s>>>(ctx->d_state, ctx->bs, covered_end, ctx->cfg.d, check_status ? 1 : 0);
+    return after_launch(ctx, "block_norm_kernel");
 }
 
 int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
@@ -249,6 +277,7 @@ int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     if (bf16) units &= ~(int64_t)1;   // bulk copies move multiples of 16 bytes
     PP.units = units;
     PP.tiles = 0;   // set by the launcher from the tile shape
+    if (ctx->bs.B > 0) fill_block_params(ctx, PP.v, units << 2);
     // Floors and up-decisions are summed as integer-valued floats: exact while n * (T + 1) <= 2^24.
     const float t_max = (float)((1 << 24) / ctx->cfg.n - 2);
     PP.fast_limit = ctx->Lf < t_max ? ctx->Lf : t_max;
@@ -262,7 +291,17 @@ int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
         std::snprintf(ctx->err, 256, "fused_pipe_kernel setup failed: %s", cudaGetErrorString(e));
         return INTSGD_ERR_CUDA;
     }
-    return after_launch(ctx, "fused_pipe_kernel");
+    const int rc = after_launch(ctx, "fused_pipe_kernel");
+    if (rc != INTSGD_OK || ctx->bs.B == 0) return rc;
+    return launch_block_norm(ctx, units << 2, true, s);
+}
+
+template <int GRAD, bool ALIGNED>
+void launch_fused_blocks_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStream_t s) {
+    if (ctx->cfg.rounding == INTSGD_ROUND_NEAREST)
+        fused_step_blocks_kernel<GRAD, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
+    else
+        fused_step_blocks_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
 
 int launch_fused(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
@@ -270,6 +309,18 @@ int launch_fused(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t
     if (want_pipe) return launch_fused_pipe(ctx, P, s);
     const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
+    if (ctx->bs.B > 0) {
+        VecParams Q = P;
+        const int64_t covered = (ctx->cfg.d >> 2) << 2;
+        fill_block_params(ctx, Q, covered);
+        if (!bf16 && aligned) launch_fused_blocks_r<INTSGD_GRAD_F32, true>(ctx, Q, grid, s);
+        else if (!bf16) launch_fused_blocks_r<INTSGD_GRAD_F32, false>(ctx, Q, grid, s);
+        else if (aligned) launch_fused_blocks_r<INTSGD_GRAD_BF16, true>(ctx, Q, grid, s);
+        else launch_fused_blocks_r<INTSGD_GRAD_BF16, false>(ctx, Q, grid, s);
+        const int rc = after_launch(ctx, "fused_step_blocks_kernel");
+        if (rc != INTSGD_OK) return rc;
+        return launch_block_norm(ctx, covered, true, s);
+    }
     if (!bf16 && aligned) launch_fused_r<INTSGD_GRAD_F32, true>(ctx, P, grid, s);
     else if (!bf16) launch_fused_r<INTSGD_GRAD_F32, false>(ctx, P, grid, s);
     else if (aligned) launch_fused_r<INTSGD_GRAD_BF16, true>(ctx, P, grid, s);
@@ -280,6 +331,20 @@ int launch_fused(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t
 int launch_exact(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
     const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
+    if (ctx->bs.B > 0) {
+        VecParams Q = P;
+        const int64_t covered = (ctx->cfg.d >> 2) << 2;
+        fill_block_params(ctx, Q, covered);
+        if (cudaMemsetAsync(ctx->bs.edge_sum, 0, sizeof(double) * ctx->bs.B, s) != cudaSuccess)
+            return fail(ctx, INTSGD_ERR_CUDA, "cudaMemsetAsync failed");
+        if (!bf16 && aligned) exact_step_blocks_kernel<INTSGD_GRAD_F32, true><<<grid, ctx->threads, 0, s>>>(Q);
+        else if (!bf16) exact_step_blocks_kernel<INTSGD_GRAD_F32, false><<<grid, ctx->threads, 0, s>>>(Q);
+        else if (aligned) exact_step_blocks_kernel<INTSGD_GRAD_BF16, true><<<grid, ctx->threads, 0, s>>>(Q);
+        else exact_step_blocks_kernel<INTSGD_GRAD_BF16, false><<<grid, ctx->threads, 0, s>>>(Q);
+        const int rc = after_launch(ctx, "exact_step_blocks_kernel");
+        if (rc != INTSGD_OK) return rc;
+        return launch_block_norm(ctx, covered, false, s);
+    }
     if (!bf16 && aligned) exact_step_kernel<INTSGD_GRAD_F32, true><<<grid, ctx->threads, 0, s>>>(P);
     else if (!bf16) exact_step_kernel<INTSGD_GRAD_F32, false><<<grid, ctx->threads, 0, s>>>(P);
     else if (aligned) exact_step_kernel<INTSGD_GRAD_BF16, true><<<grid, ctx->threads, 0, s>>>(P);
@@ -302,6 +367,18 @@ void free_staging(intsgd_ctx* ctx) {
     if (ctx->stage_agg) cudaFree(ctx->stage_agg);
     ctx->stage_x = nullptr;
     ctx->stage_agg = nullptr;
+}
+
+void free_blocks(intsgd_ctx* ctx) {
+    if (ctx->d_offsets) cudaFree(ctx->d_offsets);
+    if (ctx->bs.r) cudaFree(ctx->bs.r);            // one allocation holds every per-segment array
+    if (ctx->bs.chunk_sum) cudaFree(ctx->bs.chunk_sum);
+    ctx->d_offsets = nullptr;
+    std::memset(&ctx->bs, 0, sizeof ctx->bs);
+}
+
+int block_mode_unsupported(intsgd_ctx* ctx, const char* what) {
+    return fail(ctx, INTSGD_ERR_UNSUPPORTED, "%s is not available with block-wise scales (use intsgd_step, EXACT or FUSED)", what);
 }
 
 }  // namespace
@@ -380,6 +457,7 @@ int intsgd_destroy(intsgd_ctx* ctx) {
     if (!ctx) return INTSGD_OK;
     DeviceGuard guard(ctx->cfg.device);
     free_staging(ctx);
+    free_blocks(ctx);
     cudaFree(ctx->d_state);
     cudaFree(ctx->d_partials);
     delete ctx;
@@ -396,6 +474,7 @@ int intsgd_scale(intsgd_ctx* ctx, double eta_k, double dx2_override, void* strea
 int intsgd_sqdiff(intsgd_ctx* ctx, const float* x, const float* x_prev, void* stream) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
+    if (ctx->bs.B > 0) return block_mode_unsupported(ctx, "intsgd_sqdiff");
     bool al = true;
     int rc;
     if ((rc = check_vector(ctx, x, 4, "x", &al)) != INTSGD_OK) return rc;
@@ -416,6 +495,7 @@ int intsgd_encode(intsgd_ctx* ctx, int32_t worker, const void* grad, void* paylo
                   void* stream) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
+    if (ctx->bs.B > 0) return block_mode_unsupported(ctx, "intsgd_encode");
     if (worker < 0 || worker >= ctx->cfg.n) return fail(ctx, INTSGD_ERR_INVALID_ARG, "worker index out of range");
     if (std::isinf(alpha_override) || alpha_override <= 0.0f)
         return fail(ctx, INTSGD_ERR_INVALID_ARG, "alpha_override must be NaN (use state) or finite and > 0");
@@ -436,6 +516,7 @@ int intsgd_encode(intsgd_ctx* ctx, int32_t worker, const void* grad, void* paylo
 int intsgd_aggregate(intsgd_ctx* ctx, const void* const* payloads, float* x, int32_t* agg, void* stream) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
+    if (ctx->bs.B > 0) return block_mode_unsupported(ctx, "intsgd_aggregate");
     if (!payloads) return fail(ctx, INTSGD_ERR_INVALID_ARG, "payloads is NULL");
     bool al = true;
     int rc;
@@ -460,6 +541,7 @@ int intsgd_step(intsgd_ctx* ctx, const void* const* grads, void* const* payload_
     if (mode != INTSGD_MODE_EXACT && mode != INTSGD_MODE_TWO_KERNEL && mode != INTSGD_MODE_FUSED)
         return fail(ctx, INTSGD_ERR_INVALID_ARG, "bad mode");
     if (!grads) return fail(ctx, INTSGD_ERR_INVALID_ARG, "grads is NULL");
+    if (mode == INTSGD_MODE_TWO_KERNEL && ctx->bs.B > 0) return block_mode_unsupported(ctx, "INTSGD_MODE_TWO_KERNEL");
     if (mode == INTSGD_MODE_TWO_KERNEL && !payload_scratch)
         return fail(ctx, INTSGD_ERR_INVALID_ARG, "TWO_KERNEL mode needs payload_scratch");
     if (!(eta_k > 0.0) || !std::isfinite(eta_k)) return fail(ctx, INTSGD_ERR_INVALID_ARG, "eta_k must be finite and > 0");
@@ -584,6 +666,78 @@ int intsgd_set_state(intsgd_ctx* ctx, const intsgd_state* in) {
     h.ticket = 0;
     h.fault = 0;
     CUDA_TRY(ctx, cudaMemcpy(ctx->d_state, &h, sizeof h, cudaMemcpyHostToDevice));
+    return INTSGD_OK;
+}
+
+int intsgd_set_blocks(intsgd_ctx* ctx, int32_t num_blocks, const int64_t* offsets) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->last_stream));
+    if (num_blocks == 0) {
+        free_blocks(ctx);
+        return INTSGD_OK;
+    }
+    if (num_blocks < 0 || num_blocks > INTSGD_MAX_BLOCKS || !offsets)
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "num_blocks must be in 0..INTSGD_MAX_BLOCKS with offsets given");
+    if (offsets[0] != 0 || offsets[num_blocks] != ctx->cfg.d)
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "offsets must start at 0 and end at d");
+    for (int l = 0; l < num_blocks; ++l)
+        if (offsets[l + 1] <= offsets[l]) return fail(ctx, INTSGD_ERR_INVALID_ARG, "offsets must be strictly increasing");
+    free_blocks(ctx);
+    const size_t B = (size_t)num_blocks;
+    const size_t chunks = (size_t)((ctx->cfg.d + kChunkCoords - 1) / kChunkCoords);
+    // per-segment arrays in one allocation: r, r_new, dx2, edge_sum (double), tail_sq (8 doubles), alpha, c (float)
+    const size_t bytes = (4 * B + kMaxTail) * sizeof(double) + 2 * B * sizeof(float);
+    void* base = nullptr;
+    CUDA_TRY(ctx, cudaMalloc(&ctx->d_offsets, (B + 1) * sizeof(int64_t)));
+    cudaError_t e = cudaMalloc(&base, bytes);
+    double* chunk = nullptr;
+    if (e == cudaSuccess) e = cudaMalloc((void**)&chunk, chunks * sizeof(double));
+    if (e == cudaSuccess) e = cudaMemset(base, 0, bytes);
+    if (e == cudaSuccess) e = cudaMemset(chunk, 0, chunks * sizeof(double));
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->d_offsets, offsets, (B + 1) * sizeof(int64_t), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        if (base) cudaFree(base);
+        if (chunk) cudaFree(chunk);
+        cudaFree(ctx->d_offsets);
+        ctx->d_offsets = nullptr;
+        return fail(ctx, INTSGD_ERR_CUDA, "intsgd_set_blocks: %s", cudaGetErrorString(e));
+    }
+    double* dbl = static_cast<double*>(base);
+    ctx->bs.offsets = ctx->d_offsets;
+    ctx->bs.r = dbl;
+    ctx->bs.r_new = dbl + B;
+    ctx->bs.dx2 = dbl + 2 * B;
+    ctx->bs.edge_sum = dbl + 3 * B;
+    ctx->bs.tail_sq = dbl + 4 * B;
+    ctx->bs.alpha = reinterpret_cast<float*>(dbl + 4 * B + kMaxTail);
+    ctx->bs.c = ctx->bs.alpha + B;
+    ctx->bs.chunk_sum = chunk;
+    ctx->bs.B = num_blocks;
+    return INTSGD_OK;
+}
+
+int intsgd_get_block_state(intsgd_ctx* ctx, double* r, double* dx2, float* alpha, float* c) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    if (ctx->bs.B == 0) return fail(ctx, INTSGD_ERR_INVALID_ARG, "no block partition is set");
+    DeviceGuard guard(ctx->cfg.device);
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->last_stream));
+    const size_t B = (size_t)ctx->bs.B;
+    if (r) CUDA_TRY(ctx, cudaMemcpy(r, ctx->bs.r, B * sizeof(double), cudaMemcpyDeviceToHost));
+    if (dx2) CUDA_TRY(ctx, cudaMemcpy(dx2, ctx->bs.dx2, B * sizeof(double), cudaMemcpyDeviceToHost));
+    if (alpha) CUDA_TRY(ctx, cudaMemcpy(alpha, ctx->bs.alpha, B * sizeof(float), cudaMemcpyDeviceToHost));
+    if (c) CUDA_TRY(ctx, cudaMemcpy(c, ctx->bs.c, B * sizeof(float), cudaMemcpyDeviceToHost));
+    return INTSGD_OK;
+}
+
+int intsgd_set_block_state(intsgd_ctx* ctx, const double* r, const double* dx2) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    if (ctx->bs.B == 0) return fail(ctx, INTSGD_ERR_INVALID_ARG, "no block partition is set");
+    DeviceGuard guard(ctx->cfg.device);
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->last_stream));
+    const size_t B = (size_t)ctx->bs.B;
+    if (r) CUDA_TRY(ctx, cudaMemcpy(ctx->bs.r, r, B * sizeof(double), cudaMemcpyHostToDevice));
+    if (dx2) CUDA_TRY(ctx, cudaMemcpy(ctx->bs.dx2, dx2, B * sizeof(double), cudaMemcpyHostToDevice));
     return INTSGD_OK;
 }
 

@@ -1,0 +1,364 @@
+// Block-wise scales (Algorithm 2 of the IntSGD paper, "adaptive block quantization"): the
+// coordinates are partitioned into B contiguous blocks ("segments" below, to avoid confusion with
+// thread blocks); each has its own moving average r_{k,l}, scale alpha_{k,l} and decode factor c_l.
+//
+// The vector kernels need two things from this header:
+//  * the scale of every coordinate of a unit (UnitScale), looked up once per 32-unit chunk;
+//  * the squared step length of every segment, summed in a fixed order: a chunk (32 consecutive
+//    units = 128 coordinates, the work of one warp) that lies inside one segment stores one partial
+//    in chunk_sum[]; a chunk that straddles segments adds one partial per segment to edge_sum[]
+//    (a segment receives at most two such additions -- from the chunk holding its first and the one
+//    holding its last coordinate -- so the order of the atomics cannot change the result); the
+//    block_norm_kernel then adds everything per segment in a fixed order.
+#pragma once
+
+#include "intsgd_device.cuh"
+
+namespace intsgd {
+
+constexpr int kChunkCoords = 128;   // 32 units of 4 coordinates: one warp's unit group
+constexpr int kMaxTail = 8;
+
+// Index l with offsets[l] <= j < offsets[l + 1].
+__device__ __forceinline__ int seg_of(const BlockParams& bp, int64_t j) {
+    int lo = 0, hi = bp.B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(&bp.offsets[mid]) <= j) lo = mid;
+        else hi = mid;
+    }
+    return lo;
+}
+
+// Scales of the four coordinates of one unit.
+struct UnitScale {
+    float2 a01, a23;   // alpha of coordinates 0,1 and 2,3
+    float4 c;          // decode factors
+    int seg[4];
+};
+
+// Segment range [s_lo, s_hi] of the chunk that starts at unit `chunk_unit0` (warp-uniform).
+__device__ __forceinline__ void chunk_segments(const BlockParams& bp, int64_t chunk_unit0, int& s_lo, int& s_hi) {
+    const int64_t j_lo = chunk_unit0 << 2;
+    int64_t j_hi = j_lo + kChunkCoords;
+    if (j_hi > bp.covered_end) j_hi = bp.covered_end;
+    s_lo = seg_of(bp, j_lo);
+    s_hi = (j_hi - 1 < __ldg(&bp.offsets[s_lo + 1])) ? s_lo : seg_of(bp, j_hi - 1);
+}
+
+__device__ __forceinline__ UnitScale unit_scale(const BlockParams& bp, int64_t unit, int s_lo, int s_hi) {
+    UnitScale u;
+    if (s_lo == s_hi) {
+        const float a = __ldg(&bp.alpha[s_lo]), c = __ldg(&bp.c[s_lo]);
+        u.a01 = make_float2(a, a);
+        u.a23 = u.a01;
+        u.c = make_float4(c, c, c, c);
+        u.seg[0] = u.seg[1] = u.seg[2] = u.seg[3] = s_lo;
+        return u;
+    }
+    float a[4], c[4];
+    int s = seg_of(bp, unit << 2);
+    for (int e = 0; e < 4; ++e) {
+        const int64_t j = (unit << 2) + e;
+        while (s + 1 < bp.B && __ldg(&bp.offsets[s + 1]) <= j) ++s;
+        u.seg[e] = s;
+        a[e] = __ldg(&bp.alpha[s]);
+        c[e] = __ldg(&bp.c[s]);
+    }
+    u.a01 = make_float2(a[0], a[1]);
+    u.a23 = make_float2(a[2], a[3]);
+    u.c = make_float4(c[0], c[1], c[2], c[3]);
+    return u;
+}
+
+// Commit the squared steps of one chunk.  Must be called by all 32 lanes of a warp whose lanes own
+// consecutive units starting at chunk_unit0; lanes without a unit pass zeros.
+__device__ __forceinline__ void chunk_commit(const BlockParams& bp, int64_t chunk_unit0, int s_lo, int s_hi,
+                                             const double sq[4], const int seg[4]) {
+    const int lane = threadIdx.x & 31;
+    if (s_lo == s_hi) {
+        const double t = warp_tree(((sq[0] + sq[1]) + sq[2]) + sq[3]);
+        if (lane == 0) __stcg(&bp.chunk_sum[chunk_unit0 >> 5], t);
+        return;
+    }
+    for (int l = s_lo; l <= s_hi; ++l) {
+        double v = 0.0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (seg[e] == l) v += sq[e];
+        const double t = warp_tree(v);
+        if (lane == 0) atomicAdd(&bp.edge_sum[l], t);
+    }
+}
+
+// Squared fp32 step of one coordinate (the quantity Algorithm 2 sums per block).
+__device__ __forceinline__ float update_coord_sq(float x_old, float S_as_float, float c, double& sq) {
+    const float t = __fmul_rn(c, S_as_float);
+    const float x_new = __fsub_rn(x_old, t);
+    const float dj = __fsub_rn(x_new, x_old);
+    sq = (double)dj * (double)dj;   // exact
+    return x_new;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Per-segment state and the two small kernels of a block-wise step.
+// ---------------------------------------------------------------------------------------------
+struct BlockState {
+    const int64_t* offsets;
+    double* r;          // B: moving averages
+    double* r_new;      // B: scratch of the scale kernel
+    double* dx2;        // B: squared step lengths left by the last step
+    float* alpha;       // B
+    float* c;           // B
+    double* chunk_sum;
+    double* edge_sum;
+    double* tail_sq;
+    int32_t B;
+};
+
+// Algorithm 2, moving averages and scales, one launch of a single thread block:
+// r_l = beta r_l + (1 - beta) dx2_l;  alpha_l = eta sqrt(d_l) / sqrt(2 n r_l + eta^2 (d_l / d) eps^2);
+// c_l = eta / (n alpha_l).  All segments or none: if any scale is not finite and positive the state
+// keeps its old r and the step's vector kernels do nothing.
+__global__ void __launch_bounds__(1024) scale_blocks_kernel(DevState* st, BlockState bs, double d_total, double two_n,
+                                                            double n_as_double, double eta, double beta, double eps,
+                                                            int32_t n) {
+    int bad = 0;
+    for (int l = threadIdx.x; l < bs.B; l += blockDim.x) {
+        const double dl = (double)(bs.offsets[l + 1] - bs.offsets[l]);
+        const double a = __dmul_rn(beta, bs.r[l]);
+        const double b = __dmul_rn(__dsub_rn(1.0, beta), bs.dx2[l]);
+        const double r = __dadd_rn(a, b);
+        const double num = __dmul_rn(eta, __dsqrt_rn(dl));
+        const double two_n_r = __dmul_rn(two_n, r);
+        const double share = __ddiv_rn(dl, d_total);
+        const double guard = __dmul_rn(__dmul_rn(__dmul_rn(eta, eta), share), __dmul_rn(eps, eps));
+        const double alpha64 = __ddiv_rn(num, __dsqrt_rn(__dadd_rn(two_n_r, guard)));
+        const float alpha = __double2float_rn(alpha64);
+        const float c = __double2float_rn(__ddiv_rn(eta, __dmul_rn(n_as_double, (double)alpha)));
+        const bool ok = (alpha > 0.0f) && (alpha <= 3.402823466e+38f) && (c > 0.0f) && (c <= 3.402823466e+38f);
+        bad |= ok ? 0 : 1;
+        bs.r_new[l] = r;
+        bs.alpha[l] = alpha;
+        bs.c[l] = c;
+        bs.edge_sum[l] = 0.0;
+    }
+    const int any_bad = __syncthreads_or(bad);
+    if (!any_bad)
+        for (int l = threadIdx.x; l < bs.B; l += blockDim.x) bs.r[l] = bs.r_new[l];
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < n; ++i) st->clip_count[i] = 0;
+        st->nonfinite = 0;
+        st->agg_overflow = 0;
+        st->max_abs_agg = 0;
+        st->ticket = 0;
+        st->status = any_bad ? INTSGD_ERR_SCALE_NONFINITE : INTSGD_OK;
+        if (!any_bad) {
+            st->alpha = bs.alpha[0];
+            st->c = bs.c[0];
+        }
+    }
+}
+
+// Per-segment squared step length: thread block l adds, in a fixed order, the chunk partials that
+// lie inside segment l, the (at most two) edge partials, and the tail coordinates of the segment.
+// The block that finishes last adds the B results into state.dx2 and advances the step counter.
+__global__ void __launch_bounds__(256) block_norm_kernel(DevState* st, BlockState bs, int64_t covered_end, int64_t d,
+                                                         int32_t check_status) {
+    __shared__ double s_warp[32];
+    __shared__ bool s_last;
+    if (check_status && st->status != INTSGD_OK) return;
+    const int l = blockIdx.x;
+    const int64_t lo = bs.offsets[l];
+    int64_t hi = bs.offsets[l + 1];
+    if (hi > covered_end) hi = covered_end;
+    double v = 0.0;
+    if (lo < hi) {
+        const int64_t k0 = (lo + kChunkCoords - 1) / kChunkCoords;
+        int64_t k1 = hi / kChunkCoords;   // chunks k0 .. k1-1 end at or before hi
+        // the last, partial chunk of the covered range is interior if it starts inside the segment
+        if (hi == covered_end && (covered_end % kChunkCoords) != 0 && k1 * kChunkCoords >= lo) k1 += 1;
+        for (int64_t k = k0 + threadIdx.x; k < k1; k += blockDim.x) v += __ldcg(&bs.chunk_sum[k]);
+    }
+    double total = block_tree(v, s_warp);
+    if (threadIdx.x == 0) {
+        total += __ldcg(&bs.edge_sum[l]);
+        for (int64_t j = covered_end; j < d; ++j)
+            if (j >= bs.offsets[l] && j < bs.offsets[l + 1]) total += __ldcg(&bs.tail_sq[j - covered_end]);
+        bs.dx2[l] = total;
+        __threadfence();
+        s_last = (atomicAdd(&st->ticket, 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    double w = 0.0;
+    for (int m = threadIdx.x; m < bs.B; m += blockDim.x) w += __ldcg(&bs.dx2[m]);
+    const double sum = block_tree(w, s_warp);
+    if (threadIdx.x == 0) {
+        st->dx2 = sum;
+        st->step += 1;
+        st->ticket = 0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Direct (grid-stride) kernels with block-wise scales.  A warp owns 32 consecutive units per
+// iteration (one chunk); the loop condition is warp-uniform so that every lane reaches the shuffles.
+// ---------------------------------------------------------------------------------------------
+template <int ROUND>
+__device__ __forceinline__ int4 round_unit_scaled(float4 g, float2 a01, float2 a23, uint4 w, float Lf, u64* clip_slot,
+                                                  u64* nonfinite_slot) {
+    const float y0 = __fmul_rn(a01.x, g.x), y1 = __fmul_rn(a01.y, g.y);
+    const float y2 = __fmul_rn(a23.x, g.z), y3 = __fmul_rn(a23.y, g.w);
+    const bool in_range = (fabsf(y0) <= Lf) & (fabsf(y1) <= Lf) & (fabsf(y2) <= Lf) & (fabsf(y3) <= Lf);
+    int4 q;
+    if (in_range) {
+        q.x = round_in_range<ROUND>(y0, w.x);
+        q.y = round_in_range<ROUND>(y1, w.y);
+        q.z = round_in_range<ROUND>(y2, w.z);
+        q.w = round_in_range<ROUND>(y3, w.w);
+    } else {
+        q.x = round_checked<ROUND>(y0, w.x, Lf, clip_slot, nonfinite_slot);
+        q.y = round_checked<ROUND>(y1, w.y, Lf, clip_slot, nonfinite_slot);
+        q.z = round_checked<ROUND>(y2, w.z, Lf, clip_slot, nonfinite_slot);
+        q.w = round_checked<ROUND>(y3, w.w, Lf, clip_slot, nonfinite_slot);
+    }
+    return q;
+}
+
+// Scale and decode factor of one coordinate (tails only).
+__device__ __forceinline__ void coord_scale(const BlockParams& bp, int64_t j, float& alpha, float& c) {
+    const int s = seg_of(bp, j);
+    alpha = __ldg(&bp.alpha[s]);
+    c = __ldg(&bp.c[s]);
+}
+
+template <int GRAD, bool ALIGNED, int ROUND>
+__global__ void __launch_bounds__(512) fused_step_blocks_kernel(const __grid_constant__ VecParams P) {
+    __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
+    DevState* st = P.st;
+    if (st->status != INTSGD_OK) return;
+    counters_init(s_cnt);
+    const BlockParams& bp = P.bp;
+    const uint32_t step = st->step;
+    const int n = P.n;
+    const int lane = threadIdx.x & 31;
+    u64* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
+    ThreadAcc acc = {0.0, 0, 0u};
+
+    const int64_t full = P.d >> 2;   // == bp.covered_end / 4
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x - lane); base < full; base += stride) {
+        const int64_t unit = base + lane;
+        const bool active = unit < full;
+        int s_lo, s_hi;
+        chunk_segments(bp, base, s_lo, s_hi);
+        double sq[4] = {0.0, 0.0, 0.0, 0.0};
+        int seg[4] = {-1, -1, -1, -1};
+        if (active) {
+            const UnitScale us = unit_scale(bp, unit, s_lo, s_hi);
+            int4 S = make_int4(0, 0, 0, 0);
+#pragma unroll 4
+            for (int i = 0; i < n; ++i) {
+                const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
+                uint4 w = make_uint4(0, 0, 0, 0);
+                if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, (uint32_t)i, step, P.keys);
+                const int4 q = round_unit_scaled<ROUND>(gv, us.a01, us.a23, w, P.Lf, &s_cnt[i], nonf_slot);
+                S.x += q.x; S.y += q.y; S.z += q.z; S.w += q.w;
+            }
+            const float4 xo = load_f4<ALIGNED>(P.x, unit);
+            float4 xn;
+            xn.x = update_coord_sq(xo.x, __int2float_rn(S.x), us.c.x, sq[0]);
+            xn.y = update_coord_sq(xo.y, __int2float_rn(S.y), us.c.y, sq[1]);
+            xn.z = update_coord_sq(xo.z, __int2float_rn(S.z), us.c.z, sq[2]);
+            xn.w = update_coord_sq(xo.w, __int2float_rn(S.w), us.c.w, sq[3]);
+            store_f4<ALIGNED>(P.x, unit, xn);
+            if (P.agg) store_i4<ALIGNED>(P.agg, unit, S);
+            note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
+            note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
+        }
+        chunk_commit(bp, base, s_lo, s_hi, sq, seg);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t j = full << 2; j < P.d; ++j) {
+            float alpha, c;
+            coord_scale(bp, j, alpha, c);
+            int S = 0;
+            for (int i = 0; i < n; ++i) {
+                uint32_t word = 0;
+                if (ROUND == INTSGD_ROUND_RANDOM) {
+                    const uint4 w4 = draw_unit(j >> 2, (uint32_t)i, step, P.keys);
+                    const uint32_t wv[4] = {w4.x, w4.y, w4.z, w4.w};
+                    word = wv[j & 3];
+                }
+                const float y = __fmul_rn(alpha, grad_at<GRAD>(P.in[i], j));
+                S += round_checked<ROUND>(y, word, P.Lf, &s_cnt[i], nonf_slot);
+            }
+            double sqj;
+            P.x[j] = update_coord_sq(P.x[j], __int2float_rn(S), c, sqj);
+            if (P.agg) P.agg[j] = S;
+            note_sum(S, P.agg_limit, acc);
+            bp.tail_sq[j - bp.covered_end] = sqj;
+        }
+    }
+    counters_flush(s_cnt, st);
+    flush_sum_counters(acc, st);
+}
+
+// Exact first step with per-segment squared step lengths (Algorithm 2's Input line: x^1 is the
+// uncompressed mean step; its block norms start the moving averages).
+template <int GRAD, bool ALIGNED>
+__global__ void __launch_bounds__(512) exact_step_blocks_kernel(const __grid_constant__ VecParams P) {
+    const BlockParams& bp = P.bp;
+    const int n = P.n;
+    const float c0 = P.c_exact;
+    const int lane = threadIdx.x & 31;
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x - lane); base < full; base += stride) {
+        const int64_t unit = base + lane;
+        const bool active = unit < full;
+        int s_lo, s_hi;
+        chunk_segments(bp, base, s_lo, s_hi);
+        double sq[4] = {0.0, 0.0, 0.0, 0.0};
+        int seg[4] = {-1, -1, -1, -1};
+        if (active) {
+            float4 m = load_grad4<GRAD, ALIGNED>(P.in[0], unit);
+#pragma unroll 4
+            for (int i = 1; i < n; ++i) {
+                const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
+                m.x = __fadd_rn(m.x, gv.x); m.y = __fadd_rn(m.y, gv.y);
+                m.z = __fadd_rn(m.z, gv.z); m.w = __fadd_rn(m.w, gv.w);
+            }
+            const float4 xo = load_f4<ALIGNED>(P.x, unit);
+            float4 xn;
+            xn.x = update_coord_sq(xo.x, m.x, c0, sq[0]);
+            xn.y = update_coord_sq(xo.y, m.y, c0, sq[1]);
+            xn.z = update_coord_sq(xo.z, m.z, c0, sq[2]);
+            xn.w = update_coord_sq(xo.w, m.w, c0, sq[3]);
+            store_f4<ALIGNED>(P.x, unit, xn);
+            if (s_lo == s_hi) {
+                seg[0] = seg[1] = seg[2] = seg[3] = s_lo;
+            } else {
+                const UnitScale us = unit_scale(bp, unit, s_lo, s_hi);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
+            }
+        }
+        chunk_commit(bp, base, s_lo, s_hi, sq, seg);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t j = full << 2; j < P.d; ++j) {
+            float m = grad_at<GRAD>(P.in[0], j);
+            for (int i = 1; i < n; ++i) m = __fadd_rn(m, grad_at<GRAD>(P.in[i], j));
+            double sqj;
+            P.x[j] = update_coord_sq(P.x[j], m, c0, sqj);
+            bp.tail_sq[j - bp.covered_end] = sqj;
+        }
+    }
+}
+
+}  // namespace intsgd

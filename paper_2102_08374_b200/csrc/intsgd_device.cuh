@@ -41,6 +41,18 @@ struct PhiloxKeys {
     uint32_t k1[10];
 };
 
+// Block-wise scales (Algorithm 2); B == 0 means one scalar alpha (Algorithm 1).  See intsgd_blocks.cuh.
+struct BlockParams {
+    const int64_t* offsets;   // device, B + 1 entries, offsets[0] = 0, offsets[B] = d
+    const float* alpha;       // device, B
+    const float* c;           // device, B
+    double* chunk_sum;        // device, ceil(d / 128)
+    double* edge_sum;         // device, B (cleared when the step opens)
+    double* tail_sq;          // device, 8: squared steps of the coordinates after covered_end
+    int64_t covered_end;      // coordinates below this are handled as whole units by the launch
+    int32_t B;
+};
+
 struct VecParams {
     const void* in[INTSGD_MAX_WORKERS];   // gradients (encode / fused / exact) or payloads (aggregate)
     void* out[INTSGD_MAX_WORKERS];        // payloads (encode)
@@ -57,6 +69,7 @@ struct VecParams {
     float c_exact;                        // exact step: fp32(eta / n)
     int32_t agg_limit;                    // coordinates with |S| above this count as agg_overflow
     PhiloxKeys keys;
+    BlockParams bp;
 };
 
 // ----------------------------------------------------------------------------------------
@@ -240,16 +253,21 @@ __device__ __forceinline__ double block_tree(double v, double* s_warp) {
     return t;   // valid in thread 0
 }
 
-__device__ __forceinline__ void grid_finalize(const ThreadAcc& a, DevState* st, double* partials,
-                                              bool advance_step) {
-    __shared__ double s_warp[32];
-    __shared__ bool s_last;
+// max |S| and the int8 overflow count of the whole grid (order-independent integer atomics).
+__device__ __forceinline__ void flush_sum_counters(const ThreadAcc& a, DevState* st) {
     const int mx = __reduce_max_sync(0xFFFFFFFFu, a.max_abs);
     const unsigned ov = __reduce_add_sync(0xFFFFFFFFu, a.overflow);
     if ((threadIdx.x & 31) == 0) {
         if (mx > 0) atomicMax(&st->max_abs_agg, mx);
         if (ov) atomicAdd(&st->agg_overflow, (u64)ov);
     }
+}
+
+__device__ __forceinline__ void grid_finalize(const ThreadAcc& a, DevState* st, double* partials,
+                                              bool advance_step) {
+    __shared__ double s_warp[32];
+    __shared__ bool s_last;
+    flush_sum_counters(a, st);
     const double block_sum = block_tree(a.dx2, s_warp);
     if (threadIdx.x == 0) {
         __stcg(&partials[blockIdx.x], block_sum);

@@ -12,6 +12,7 @@
 // (unaligned pointers, larger d) runs in fused_step_kernel.
 #pragma once
 
+#include "intsgd_blocks.cuh"
 #include "intsgd_device.cuh"
 
 namespace intsgd {
@@ -81,9 +82,9 @@ struct UnitAcc {
 };
 
 template <int ROUND>
-__device__ __forceinline__ void consume_unit(float4 g, float2 alpha2, uint4 w, UnitAcc& u) {
-    const float2 y01 = __fmul2_rn(alpha2, make_float2(g.x, g.y));
-    const float2 y23 = __fmul2_rn(alpha2, make_float2(g.z, g.w));
+__device__ __forceinline__ void consume_unit(float4 g, float2 alpha01, float2 alpha23, uint4 w, UnitAcc& u) {
+    const float2 y01 = __fmul2_rn(alpha01, make_float2(g.x, g.y));
+    const float2 y23 = __fmul2_rn(alpha23, make_float2(g.z, g.w));
     u.m = absmax3_nan(u.m, y01.x, y01.y);
     u.m = absmax3_nan(u.m, y23.x, y23.y);
     if (ROUND == INTSGD_ROUND_NEAREST) {
@@ -107,7 +108,8 @@ __device__ __forceinline__ void consume_unit(float4 g, float2 alpha2, uint4 w, U
 // Exact redo of one unit from global memory with the full clipping rule and the counters (rare:
 // some |alpha g| outside the fast range, or a NaN/Inf).  The fast path has counted nothing.
 template <int GRAD, int ROUND>
-__device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float alpha, uint32_t step, u64* s_cnt) {
+__device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float4 alpha4, uint32_t step, u64* s_cnt) {
+    const float av[4] = {alpha4.x, alpha4.y, alpha4.z, alpha4.w};
     int S[4] = {0, 0, 0, 0};
     for (int i = 0; i < P.n; ++i) {
         const float4 g = load_grad4<GRAD, true>(P.in[i], unit);
@@ -116,7 +118,7 @@ __device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float a
         const float gv[4] = {g.x, g.y, g.z, g.w};
         const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
         for (int e = 0; e < 4; ++e) {
-            const float y = __fmul_rn(alpha, gv[e]);
+            const float y = __fmul_rn(av[e], gv[e]);
             S[e] += round_checked<ROUND>(y, wv[e], P.Lf, &s_cnt[i], &s_cnt[INTSGD_MAX_WORKERS]);
         }
     }
@@ -181,7 +183,7 @@ __device__ __forceinline__ float4 lds_unit(const unsigned char* tile, int c) {
 // ---- the kernel ----------------------------------------------------------------------------------
 // NC consumer threads + one producer warp.  A tile is NC * UPT units; consumer c owns units
 // c, c + NC, ... of the tile.  G worker tiles per stage, NS stages.
-template <int GRAD, int ROUND, int NC, int UPT, int G, int NS>
+template <int GRAD, int ROUND, bool BLOCKS, int NC, int UPT, int G, int NS>
 __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_constant__ PipeParams PP) {
     constexpr int kUnitBytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
     constexpr int kTileUnits = NC * UPT;
@@ -243,15 +245,18 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
     } else {
         // ------------------------------- consumers --------------------------------------------
         const int c = threadIdx.x;
+        const int lane = c & 31;
         const float alpha = st->alpha, cdec = st->c;
         const uint32_t step = st->step;
-        const float2 alpha2 = make_float2(alpha, alpha);
+        const BlockParams& bp = P.bp;
         uint32_t s = 0, phase = 0;
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             const int64_t unit0 = tile * kTileUnits + c;
             float4 xo[UPT];
             PhiloxThreadPart tp[UPT];
             UnitAcc ua[UPT];
+            float2 a01[UPT], a23[UPT];
+            int s_lo[UPT], s_hi[UPT];
             bool active[UPT];
 #pragma unroll
             for (int k = 0; k < UPT; ++k) {
@@ -264,9 +269,23 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 ua[k].F01 = make_float2(0.f, 0.f);
                 ua[k].F23 = make_float2(0.f, 0.f);
                 ua[k].m = 0.0f;
+                a01[k] = make_float2(alpha, alpha);
+                a23[k] = a01[k];
+                s_lo[k] = s_hi[k] = 0;
+                if (BLOCKS) {
+                    // the warp's 32 units form one chunk; chunks past the covered range are never committed
+                    if (unit - lane < PP.units) chunk_segments(bp, unit - lane, s_lo[k], s_hi[k]);
+                    if (active[k]) {
+                        const UnitScale us = unit_scale(bp, unit, s_lo[k], s_hi[k]);
+                        a01[k] = us.a01;
+                        a23[k] = us.a23;
+                    }
+                }
             }
             for (int g0 = 0; g0 < n; g0 += G) {
-                if (!mbar_wait(&full_bar[s], phase)) { ok = false; break; }
+                bool arrived = mbar_wait(&full_bar[s], phase);
+                if (BLOCKS) arrived = __all_sync(0xFFFFFFFFu, arrived);   // keep the warp together for the shuffles below
+                if (!arrived) { ok = false; break; }
                 const unsigned char* src = smem + (size_t)s * G * kTileBytes;
                 const int gw = (n - g0 < G) ? (n - g0) : G;
                 if (active[UPT - 1] && gw == G) {
@@ -279,7 +298,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
                             uint4 rw = make_uint4(0, 0, 0, 0);
                             if (ROUND == INTSGD_ROUND_RANDOM) rw = philox_finish(tp[k], e, P.keys);
-                            consume_unit<ROUND>(gv, alpha2, rw, ua[k]);
+                            consume_unit<ROUND>(gv, a01[k], a23[k], rw, ua[k]);
                         }
                     }
                 } else {
@@ -291,7 +310,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
                             uint4 rw = make_uint4(0, 0, 0, 0);
                             if (ROUND == INTSGD_ROUND_RANDOM) rw = philox_finish(tp[k], e, P.keys);
-                            consume_unit<ROUND>(gv, alpha2, rw, ua[k]);
+                            consume_unit<ROUND>(gv, a01[k], a23[k], rw, ua[k]);
                         }
                     }
                 }
@@ -301,14 +320,44 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
             if (!ok) break;
 #pragma unroll
             for (int k = 0; k < UPT; ++k) {
-                if (!active[k]) continue;
                 const int64_t unit = unit0 + (int64_t)k * NC;
+                if (BLOCKS) {
+                    if (unit - lane >= PP.units) continue;   // warp-uniform: this chunk does not exist
+                    double sq[4] = {0.0, 0.0, 0.0, 0.0};
+                    int seg[4] = {-1, -1, -1, -1};
+                    if (active[k]) {
+                        const UnitScale us = unit_scale(bp, unit, s_lo[k], s_hi[k]);
+                        int4 S;
+                        float4 Sf;
+                        if (ua[k].m <= PP.fast_limit) {
+                            Sf = make_float4(ua[k].F01.x, ua[k].F01.y, ua[k].F23.x, ua[k].F23.y);
+                            S = make_int4(__float2int_rn(Sf.x), __float2int_rn(Sf.y), __float2int_rn(Sf.z), __float2int_rn(Sf.w));
+                        } else {
+                            S = redo_unit<GRAD, ROUND>(P, unit, make_float4(us.a01.x, us.a01.y, us.a23.x, us.a23.y), step, s_cnt);
+                            Sf = make_float4(__int2float_rn(S.x), __int2float_rn(S.y), __int2float_rn(S.z), __int2float_rn(S.w));
+                        }
+                        float4 xn;
+                        xn.x = update_coord_sq(xo[k].x, Sf.x, us.c.x, sq[0]);
+                        xn.y = update_coord_sq(xo[k].y, Sf.y, us.c.y, sq[1]);
+                        xn.z = update_coord_sq(xo[k].z, Sf.z, us.c.z, sq[2]);
+                        xn.w = update_coord_sq(xo[k].w, Sf.w, us.c.w, sq[3]);
+                        store_f4<true>(P.x, unit, xn);
+                        if (P.agg) store_i4<true>(P.agg, unit, S);
+                        note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
+                        note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
+                    }
+                    chunk_commit(bp, unit - lane, s_lo[k], s_hi[k], sq, seg);
+                    continue;
+                }
+                if (!active[k]) continue;
                 int4 S;
                 if (ua[k].m <= PP.fast_limit) {
                     S = make_int4(__float2int_rn(ua[k].F01.x), __float2int_rn(ua[k].F01.y),
                                   __float2int_rn(ua[k].F23.x), __float2int_rn(ua[k].F23.y));
                 } else {
-                    S = redo_unit<GRAD, ROUND>(P, unit, alpha, step, s_cnt);
+                    S = redo_unit<GRAD, ROUND>(P, unit, make_float4(alpha, alpha, alpha, alpha), step, s_cnt);
                 }
                 float4 xn;
                 xn.x = update_coord(xo[k].x, S.x, cdec, acc.dx2);
@@ -327,6 +376,8 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         if (blockIdx.x == 0 && c == 0 && ok) {
             const int64_t j0 = PP.units << 2;
             for (int64_t j = j0; j < P.d; ++j) {
+                float aj = alpha, cj = cdec;
+                if (BLOCKS) coord_scale(bp, j, aj, cj);
                 int S = 0;
                 for (int i = 0; i < n; ++i) {
                     uint32_t word = 0;
@@ -335,16 +386,25 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                         const uint32_t wv[4] = {w4.x, w4.y, w4.z, w4.w};
                         word = wv[j & 3];
                     }
-                    const float y = __fmul_rn(alpha, grad_at<GRAD>(P.in[i], j));
+                    const float y = __fmul_rn(aj, grad_at<GRAD>(P.in[i], j));
                     S += round_checked<ROUND>(y, word, P.Lf, &s_cnt[i], &s_cnt[INTSGD_MAX_WORKERS]);
                 }
-                apply_coord(P, j, S, cdec, acc);
+                if (BLOCKS) {
+                    double sqj;
+                    P.x[j] = update_coord_sq(P.x[j], __int2float_rn(S), cj, sqj);
+                    if (P.agg) P.agg[j] = S;
+                    note_sum(S, P.agg_limit, acc);
+                    bp.tail_sq[j - bp.covered_end] = sqj;
+                } else {
+                    apply_coord(P, j, S, cdec, acc);
+                }
             }
         }
     }
     counters_flush(s_cnt, st);   // includes a __syncthreads()
     if (threadIdx.x == 0 && s_fault) atomicExch(&st->fault, 1);
-    grid_finalize(acc, st, P.partials, true);
+    if (BLOCKS) flush_sum_counters(acc, st);   // the per-segment norms are finished by block_norm_kernel
+    else grid_finalize(acc, st, P.partials, true);
 }
 
 }  // namespace intsgd
