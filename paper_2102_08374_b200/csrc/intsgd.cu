@@ -5,6 +5,7 @@
 #include <cstring>
 #include <limits>
 #include <new>
+#include <vector>
 
 #include "intsgd_kernels.cuh"
 #include "intsgd_pipe.cuh"
@@ -30,6 +31,8 @@ struct intsgd_ctx {
     // block-wise scales (Algorithm 2); bs.B == 0 means one scalar alpha
     BlockState bs;
     int64_t* d_offsets;
+    NormPlan plan[2];     // [0]: covered range of the direct kernels and fp32; [1]: bf16 pipelined (even units)
+    void* d_plan_mem[2];
     // device staging for intsgd_step_host (allocated on first use)
     void* stage_grads[INTSGD_MAX_WORKERS];
     float* stage_x;
@@ -264,7 +267,14 @@ void fill_block_params(const intsgd_ctx* ctx, VecParams& P, int64_t covered_end)
 
 // Finishes a block-wise step: per-segment squared step lengths, total, step counter.
 int launch_block_norm(intsgd_ctx* ctx, int64_t covered_end, bool check_status, cudaStream_t s) {
-    block_norm_kernel<<<ctx->bs.B, 256, 0, s>>>(ctx->d_state, ctx->bs, covered_end, ctx->cfg.d, check_status ? 1 : 0);
+    const NormPlan& plan = (ctx->plan[0].covered_end == covered_end) ? ctx->plan[0] : ctx->plan[1];
+    if (plan.covered_end != covered_end) return fail(ctx, INTSGD_ERR_CUDA, "internal: no reduction plan for this launch");
+    if (plan.num_slices > 0) {
+        block_norm_slices_kernel<<<plan.num_slices, 256, 0, s>>>(ctx->d_state, ctx->bs, plan, check_status ? 1 : 0);
+        const int rc = after_launch(ctx, "block_norm_slices_kernel");
+        if (rc != INTSGD_OK) return rc;
+    }
+    block_norm_kernel<<<ctx->bs.B, 128, 0, s>>>(ctx->d_state, ctx->bs, plan, ctx->cfg.d, check_status ? 1 : 0);
     return after_launch(ctx, "block_norm_kernel");
 }
 
@@ -369,7 +379,55 @@ void free_staging(intsgd_ctx* ctx) {
     ctx->stage_agg = nullptr;
 }
 
+// Host side of NormPlan: slices of the chunk range of every segment for a given covered range.
+cudaError_t build_norm_plan(const int64_t* offsets, int B, int64_t covered_end, NormPlan* plan, void** mem) {
+    std::vector<int64_t> k0, k1;
+    std::vector<int32_t> seg_slice(B + 1, 0);
+    for (int l = 0; l < B; ++l) {
+        seg_slice[l] = (int32_t)k0.size();
+        const int64_t lo = offsets[l];
+        const int64_t hi = offsets[l + 1] < covered_end ? offsets[l + 1] : covered_end;
+        if (lo >= hi) continue;
+        const int64_t first = (lo + kChunkCoords - 1) / kChunkCoords;
+        int64_t last = hi / kChunkCoords;   // chunks first .. last-1 end at or before hi
+        // the partial chunk that ends the covered range is interior if it starts inside the segment
+        if (hi == covered_end && (covered_end % kChunkCoords) != 0 && last * kChunkCoords >= lo) last += 1;
+        for (int64_t k = first; k < last; k += kSliceChunks) {
+            k0.push_back(k);
+            k1.push_back(k + kSliceChunks < last ? k + kSliceChunks : last);
+        }
+    }
+    seg_slice[B] = (int32_t)k0.size();
+    const size_t ns = k0.size();
+    const size_t bytes = (2 * ns) * sizeof(int64_t) + ns * sizeof(double) + (size_t)(B + 1) * sizeof(int32_t);
+    char* base = nullptr;
+    cudaError_t e = cudaMalloc((void**)&base, bytes);
+    if (e != cudaSuccess) return e;
+    int64_t* d_k0 = reinterpret_cast<int64_t*>(base);
+    int64_t* d_k1 = d_k0 + ns;
+    double* d_sum = reinterpret_cast<double*>(d_k1 + ns);
+    int32_t* d_seg = reinterpret_cast<int32_t*>(d_sum + ns);
+    if (ns) e = cudaMemcpy(d_k0, k0.data(), ns * sizeof(int64_t), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && ns) e = cudaMemcpy(d_k1, k1.data(), ns * sizeof(int64_t), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(d_seg, seg_slice.data(), (size_t)(B + 1) * sizeof(int32_t), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { cudaFree(base); return e; }
+    plan->k0 = d_k0;
+    plan->k1 = d_k1;
+    plan->seg_slice = d_seg;
+    plan->slice_sum = d_sum;
+    plan->covered_end = covered_end;
+    plan->num_slices = (int32_t)ns;
+    *mem = base;
+    return cudaSuccess;
+}
+
 void free_blocks(intsgd_ctx* ctx) {
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->d_plan_mem[i]) cudaFree(ctx->d_plan_mem[i]);
+        ctx->d_plan_mem[i] = nullptr;
+        std::memset(&ctx->plan[i], 0, sizeof ctx->plan[i]);
+        ctx->plan[i].covered_end = -1;
+    }
     if (ctx->d_offsets) cudaFree(ctx->d_offsets);
     if (ctx->bs.r) cudaFree(ctx->bs.r);            // one allocation holds every per-segment array
     if (ctx->bs.chunk_sum) cudaFree(ctx->bs.chunk_sum);
@@ -426,6 +484,7 @@ int intsgd_create(intsgd_ctx** out, const intsgd_config* cfg) {
     ctx->keys = make_keys(cfg->seed);
     ctx->tab = make_worker_table(ctx->keys);
     ctx->fused_path = 0;
+    ctx->plan[0].covered_end = ctx->plan[1].covered_end = -1;
     ctx->threads = kDefaultThreads;
     ctx->blocks_per_sm = kDefaultBlocksPerSm;
 
@@ -696,7 +755,16 @@ int intsgd_set_blocks(intsgd_ctx* ctx, int32_t num_blocks, const int64_t* offset
     if (e == cudaSuccess) e = cudaMemset(base, 0, bytes);
     if (e == cudaSuccess) e = cudaMemset(chunk, 0, chunks * sizeof(double));
     if (e == cudaSuccess) e = cudaMemcpy(ctx->d_offsets, offsets, (B + 1) * sizeof(int64_t), cudaMemcpyHostToDevice);
+    // covered ranges: whole units of 4 (direct kernels, fp32 pipelined) and pairs of units (bf16 pipelined)
+    const int64_t cov0 = (ctx->cfg.d >> 2) << 2, cov1 = (ctx->cfg.d >> 3) << 3;
+    if (e == cudaSuccess) e = build_norm_plan(offsets, num_blocks, cov0, &ctx->plan[0], &ctx->d_plan_mem[0]);
+    if (e == cudaSuccess && cov1 != cov0) e = build_norm_plan(offsets, num_blocks, cov1, &ctx->plan[1], &ctx->d_plan_mem[1]);
     if (e != cudaSuccess) {
+        for (int i = 0; i < 2; ++i) {
+            if (ctx->d_plan_mem[i]) cudaFree(ctx->d_plan_mem[i]);
+            ctx->d_plan_mem[i] = nullptr;
+            ctx->plan[i].covered_end = -1;
+        }
         if (base) cudaFree(base);
         if (chunk) cudaFree(chunk);
         cudaFree(ctx->d_offsets);

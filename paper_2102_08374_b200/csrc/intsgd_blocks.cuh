@@ -8,8 +8,8 @@
 //    units = 128 coordinates, the work of one warp) that lies inside one segment stores one partial
 //    in chunk_sum[]; a chunk that straddles segments adds one partial per segment to edge_sum[]
 //    (a segment receives at most two such additions -- from the chunk holding its first and the one
-//    holding its last coordinate -- so the order of the atomics cannot change the result); the
-//    block_norm_kernel then adds everything per segment in a fixed order.
+//    holding its last coordinate -- so the order of the atomics cannot change the result); the two
+//    block_norm kernels then add everything per segment in a fixed order.
 #pragma once
 
 #include "intsgd_device.cuh"
@@ -160,31 +160,48 @@ __global__ void __launch_bounds__(1024) scale_blocks_kernel(DevState* st, BlockS
     }
 }
 
-// Per-segment squared step length: thread block l adds, in a fixed order, the chunk partials that
-// lie inside segment l, the (at most two) edge partials, and the tail coordinates of the segment.
-// The block that finishes last adds the B results into state.dx2 and advances the step counter.
-__global__ void __launch_bounds__(256) block_norm_kernel(DevState* st, BlockState bs, int64_t covered_end, int64_t d,
+// Reduction plan for the per-segment norms, built on the host when the partition is set: the chunk
+// partials that lie inside a segment are cut into slices of at most kSliceChunks chunks, so that long
+// segments are summed by many thread blocks.  Slice w covers chunks [k0[w], k1[w]) of one segment;
+// segment l owns slices [seg_slice[l], seg_slice[l + 1]).
+constexpr int kSliceChunks = 1024;
+struct NormPlan {
+    const int64_t* k0;         // device, num_slices
+    const int64_t* k1;         // device, num_slices
+    const int32_t* seg_slice;  // device, B + 1
+    double* slice_sum;         // device, num_slices
+    int64_t covered_end;
+    int32_t num_slices;
+};
+
+// Pass 1: one thread block per slice, fixed summation order.
+__global__ void __launch_bounds__(256) block_norm_slices_kernel(const DevState* st, BlockState bs, NormPlan plan,
+                                                                int32_t check_status) {
+    __shared__ double s_warp[32];
+    if (check_status && st->status != INTSGD_OK) return;
+    const int w = blockIdx.x;
+    double v = 0.0;
+    for (int64_t k = plan.k0[w] + threadIdx.x; k < plan.k1[w]; k += blockDim.x) v += __ldcg(&bs.chunk_sum[k]);
+    const double t = block_tree(v, s_warp);
+    if (threadIdx.x == 0) plan.slice_sum[w] = t;
+}
+
+// Pass 2: thread block l adds the slices of segment l in order, then the (at most two) edge partials
+// and the segment's tail coordinates.  The block that finishes last adds the B results into
+// state.dx2 and advances the step counter.
+__global__ void __launch_bounds__(128) block_norm_kernel(DevState* st, BlockState bs, NormPlan plan, int64_t d,
                                                          int32_t check_status) {
     __shared__ double s_warp[32];
     __shared__ bool s_last;
     if (check_status && st->status != INTSGD_OK) return;
     const int l = blockIdx.x;
-    const int64_t lo = bs.offsets[l];
-    int64_t hi = bs.offsets[l + 1];
-    if (hi > covered_end) hi = covered_end;
     double v = 0.0;
-    if (lo < hi) {
-        const int64_t k0 = (lo + kChunkCoords - 1) / kChunkCoords;
-        int64_t k1 = hi / kChunkCoords;   // chunks k0 .. k1-1 end at or before hi
-        // the last, partial chunk of the covered range is interior if it starts inside the segment
-        if (hi == covered_end && (covered_end % kChunkCoords) != 0 && k1 * kChunkCoords >= lo) k1 += 1;
-        for (int64_t k = k0 + threadIdx.x; k < k1; k += blockDim.x) v += __ldcg(&bs.chunk_sum[k]);
-    }
+    for (int w = plan.seg_slice[l] + threadIdx.x; w < plan.seg_slice[l + 1]; w += blockDim.x) v += __ldcg(&plan.slice_sum[w]);
     double total = block_tree(v, s_warp);
     if (threadIdx.x == 0) {
         total += __ldcg(&bs.edge_sum[l]);
-        for (int64_t j = covered_end; j < d; ++j)
-            if (j >= bs.offsets[l] && j < bs.offsets[l + 1]) total += __ldcg(&bs.tail_sq[j - covered_end]);
+        for (int64_t j = plan.covered_end; j < d; ++j)
+            if (j >= bs.offsets[l] && j < bs.offsets[l + 1]) total += __ldcg(&bs.tail_sq[j - plan.covered_end]);
         bs.dx2[l] = total;
         __threadfence();
         s_last = (atomicAdd(&st->ticket, 1u) == gridDim.x - 1);
@@ -192,9 +209,9 @@ __global__ void __launch_bounds__(256) block_norm_kernel(DevState* st, BlockStat
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    double w = 0.0;
-    for (int m = threadIdx.x; m < bs.B; m += blockDim.x) w += __ldcg(&bs.dx2[m]);
-    const double sum = block_tree(w, s_warp);
+    double w2 = 0.0;
+    for (int m = threadIdx.x; m < bs.B; m += blockDim.x) w2 += __ldcg(&bs.dx2[m]);
+    const double sum = block_tree(w2, s_warp);
     if (threadIdx.x == 0) {
         st->dx2 = sum;
         st->step += 1;
