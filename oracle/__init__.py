@@ -81,6 +81,11 @@ def lib() -> C.CDLL:
                                       C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                       f64p, u64p, u64p, u64p, i32p]
         L.orc_step_window.restype = None
+        L.orc_diana_step_window.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64, C.c_int64,
+                                            C.c_float, C.c_float, C.c_float, C.c_float, C.c_int64, C.c_int,
+                                            C.c_int, C.c_uint64, C.c_uint32, C.POINTER(C.c_void_p), C.c_void_p,
+                                            C.c_void_p, C.c_void_p, f64p, u64p, u64p, u64p, i32p]
+        L.orc_diana_step_window.restype = None
     return _lib
 
 
@@ -329,3 +334,63 @@ class OracleIntSGDBlocks:
         return dict(agg=agg, dx2=list(new_dx2), r=list(self.r), alpha64=[t[1] for t in sc],
                     alpha=[t[2] for t in sc], c=[t[3] for t in sc], clip_count=clip, nonfinite=nonf,
                     agg_overflow=ovf, max_abs_agg=mx)
+
+
+def diana_factors(n, alpha, eta):
+    """fp32 factors of an IntDIANA step for a given fp32 alpha: 1/alpha, 1/(n alpha), eta."""
+    a = float(np.float32(alpha))
+    return np.float32(1.0 / a), np.float32(1.0 / (float(n) * a)), np.float32(eta)
+
+
+def diana_step_window(grads, h_local, h_global, x, alpha, eta, *, step, seed, j0=0, clip_limit=None,
+                      payload_dtype=PAYLOAD_I32, rounding=ROUND_RANDOM, want_agg=True):
+    """One IntDIANA step (Algorithm 3) on coordinates [j0, j0 + len(x)) with alpha given.
+
+    Updates h_local[i], h_global and x in place; returns agg, dx2 and the counters."""
+    grads = [np.ascontiguousarray(g) for g in grads]
+    n, count = len(grads), x.shape[0]
+    if clip_limit is None:
+        clip_limit = default_clip_limit(n, payload_dtype)
+    ainv, cn, eta32 = diana_factors(n, alpha, eta)
+    agg = np.empty(count, dtype=np.int32) if want_agg else None
+    clip = (C.c_uint64 * n)()
+    dx2, nonf, ovf, mx = C.c_double(), C.c_uint64(0), C.c_uint64(0), C.c_int32(0)
+    for h in list(h_local) + [h_global, x]:
+        assert h.dtype == np.float32 and h.flags.c_contiguous and h.shape[0] == count
+    lib().orc_diana_step_window(_ptr_array(grads), _grad_dtype(grads[0]), n, j0, count, float(np.float32(alpha)),
+                                float(ainv), float(cn), float(eta32), int(clip_limit), payload_dtype, rounding,
+                                seed, step, _ptr_array(h_local), _ptr(h_global), _ptr(x), _ptr(agg),
+                                C.byref(dx2), clip, C.byref(nonf), C.byref(ovf), C.byref(mx))
+    return dict(agg=agg, dx2=dx2.value, clip_count=[int(v) for v in clip], nonfinite=nonf.value,
+                agg_overflow=ovf.value, max_abs_agg=mx.value)
+
+
+class OracleIntDIANA:
+    """Algorithm 3 as a state machine.  Step 0 is the exact mean step with h_i = h = 0; later steps
+    use the scale rule of the context (Algorithm 3 prints its beta = 0, eps = 0 case,
+    alpha_k = eta sqrt(d) / (sqrt(2n) ||x^k - x^{k-1}||))."""
+
+    def __init__(self, n, d, *, beta=0.0, eps=0.0, seed=0, payload_dtype=PAYLOAD_I32, clip_limit=None,
+                 rounding=ROUND_RANDOM):
+        self.n, self.d, self.beta, self.eps, self.seed = n, d, beta, eps, seed
+        self.payload_dtype, self.rounding = payload_dtype, rounding
+        self.clip_limit = default_clip_limit(n, payload_dtype) if not clip_limit else clip_limit
+        self.h_local = [np.zeros(d, dtype=np.float32) for _ in range(n)]
+        self.h_global = np.zeros(d, dtype=np.float32)
+        self.r, self.dx2, self.step = 0.0, 0.0, 0
+
+    def exact_step(self, grads, x, eta):
+        self.dx2 = exact_step(grads, x, eta)
+        self.step += 1
+        return dict(dx2=self.dx2)
+
+    def int_step(self, grads, x, eta, *, alpha=None, want_agg=True):
+        r, a64, a32, c32 = scale(self.d, self.n, eta, self.beta, self.eps, self.r, self.dx2)
+        self.r = r
+        out = diana_step_window(grads, self.h_local, self.h_global, x, a32 if alpha is None else alpha, eta,
+                                step=self.step, seed=self.seed, clip_limit=self.clip_limit,
+                                payload_dtype=self.payload_dtype, rounding=self.rounding, want_agg=want_agg)
+        self.dx2 = out["dx2"]
+        self.step += 1
+        out.update(r=r, alpha64=a64, alpha=a32)
+        return out

@@ -304,4 +304,51 @@ void orc_step_window(const void* const* grads, int grad_dtype, int32_t n, int64_
     *dx2_out = dx2;
 }
 
+// ---- IntDIANA (Algorithm 3): compress gradient differences ---------------------------------
+// Worker i rounds alpha (g_i - h_i); its shift moves by the decoded message,
+// h_i <- h_i + (1/alpha) Int(alpha (g_i - h_i)) (the proof of the IntDIANA theorem defines
+// Q(g_i) = (1/alpha) Int(alpha (g_i - h_i)) for this line); the estimator and the new global
+// shift are the same vector, g~ = h + (1/(n alpha)) sum_i Int(...); x <- x - eta g~.
+// fp32 steps, each rounded once: v = g - h_i; y = alpha v; q = clip(Int(y));
+// h_i = h_i + ainv * float(q); t = cn * float(S); gt = h + t; x = x - eta32 * gt.
+// ainv = fp32(1/alpha), cn = fp32(1/(n alpha)), eta32 = fp32(eta) are given by the caller.
+void orc_diana_step_window(const void* const* grads, int grad_dtype, int32_t n, int64_t j0, int64_t count,
+                           float alpha, float ainv, float cn, float eta32, int64_t L, int payload_dtype,
+                           int rounding, uint64_t seed, uint32_t step, float* const* h_local, float* h_global,
+                           float* x, int32_t* agg, double* dx2_out, uint64_t* clip_count,
+                           uint64_t* nonfinite_count, uint64_t* agg_overflow, int32_t* max_abs_agg) {
+    const float Lf = limit_as_float(L);
+    double dx2 = 0.0;
+    for (int64_t t = 0; t < count; ++t) {
+        int32_t S = 0;
+        for (int32_t i = 0; i < n; ++i) {
+            const float g = load_grad(grads[i], grad_dtype, t);
+            const float v = g - h_local[i][t];
+            const float y = alpha * v;
+            float u = 0.0f;
+            if (rounding == 0) u = uniform_from_word(draw_word(seed, step, (uint32_t)i, (uint64_t)(j0 + t)));
+            const Rounded r = round_and_clip(y, u, Lf, rounding);
+            if (r.clipped) clip_count[i] += 1;
+            if (r.nonfinite) *nonfinite_count += 1;
+            const float dq = ainv * (float)r.q;
+            h_local[i][t] = h_local[i][t] + dq;
+            S += r.q;
+        }
+        const int32_t mag = S < 0 ? -S : S;
+        if (payload_dtype == 1 && mag > 127) *agg_overflow += 1;
+        if (mag > *max_abs_agg) *max_abs_agg = mag;
+        if (agg) agg[t] = S;
+        const float dec = cn * (float)S;
+        const float gt = h_global[t] + dec;
+        h_global[t] = gt;
+        const float stepv = eta32 * gt;
+        const float x_old = x[t];
+        const float x_new = x_old - stepv;
+        const float dj = x_new - x_old;
+        dx2 += (double)dj * (double)dj;
+        x[t] = x_new;
+    }
+    *dx2_out = dx2;
+}
+
 }  // extern "C"
