@@ -147,6 +147,19 @@ int intsgd_aggregate(intsgd_ctx* ctx, const void* const* payloads, float* x, int
 int intsgd_step(intsgd_ctx* ctx, const void* const* grads, void* const* payload_scratch,
                 float* x, int32_t* agg, double eta_k, int32_t mode, void* stream);
 
+/* One IntDIANA step (Algorithm 3: IntSGD on gradient differences, for heterogeneous data):
+ *     q_i  = clip(Int(alpha_k (g_i - h_i)))          h_i <- h_i + (1/alpha_k) q_i
+ *     g~   = h + (1/(n alpha_k)) sum_i q_i           h <- g~         x <- x - eta_k g~
+ * (the shift update uses Q(g_i) = (1/alpha) Int(alpha (g_i - h_i)), as the proof of the IntDIANA
+ * theorem defines it).  alpha_k comes from the context's scale rule; Algorithm 3 prints its
+ * beta = 0, eps = 0 case.  fp32 steps, each rounded once: v = g - h_i; y = alpha v;
+ * h_i += fp32(1/alpha) * float(q); t = fp32(1/(n alpha)) * float(S); g~ = h + t; x -= fp32(eta) * g~.
+ * h_local: HOST array of n device pointers to float[d] (read and written); h_global: device float[d]
+ * (read and written); both start at zero after the exact first step (intsgd_step, MODE_EXACT).
+ * Same counters, dx2 and step bookkeeping as intsgd_step.  Not available with a block partition. */
+int intsgd_diana_step(intsgd_ctx* ctx, const void* const* grads, float* const* h_local, float* h_global, float* x,
+                      int32_t* agg, double eta_k, void* stream);
+
 /* The same step for a caller whose buffers are in HOST memory (pinned memory recommended):
  * copies the n gradients and x to device staging buffers owned by the context (allocated on
  * first use: n*d gradient values + d floats + d int32), runs intsgd_step, copies x (and agg if

@@ -7,6 +7,7 @@
 #include <new>
 #include <vector>
 
+#include "intsgd_diana.cuh"
 #include "intsgd_kernels.cuh"
 #include "intsgd_pipe.cuh"
 
@@ -338,6 +339,23 @@ int launch_fused(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t
     return after_launch(ctx, "fused_step_kernel");
 }
 
+template <int GRAD, bool ALIGNED>
+void launch_diana_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStream_t s) {
+    if (ctx->cfg.rounding == INTSGD_ROUND_NEAREST)
+        diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
+    else
+        diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
+}
+int launch_diana(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
+    const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
+    const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
+    if (!bf16 && aligned) launch_diana_r<INTSGD_GRAD_F32, true>(ctx, P, grid, s);
+    else if (!bf16) launch_diana_r<INTSGD_GRAD_F32, false>(ctx, P, grid, s);
+    else if (aligned) launch_diana_r<INTSGD_GRAD_BF16, true>(ctx, P, grid, s);
+    else launch_diana_r<INTSGD_GRAD_BF16, false>(ctx, P, grid, s);
+    return after_launch(ctx, "diana_step_kernel");
+}
+
 int launch_exact(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
     const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
@@ -645,6 +663,35 @@ int intsgd_step(intsgd_ctx* ctx, const void* const* grads, void* const* payload_
     A.x = x;
     A.agg = agg;
     return launch_aggregate(ctx, A, al_agg, s);
+}
+
+int intsgd_diana_step(intsgd_ctx* ctx, const void* const* grads, float* const* h_local, float* h_global, float* x,
+                      int32_t* agg, double eta_k, void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (ctx->bs.B > 0) return block_mode_unsupported(ctx, "intsgd_diana_step");
+    if (!grads || !h_local) return fail(ctx, INTSGD_ERR_INVALID_ARG, "grads / h_local is NULL");
+    if (!(eta_k > 0.0) || !std::isfinite(eta_k)) return fail(ctx, INTSGD_ERR_INVALID_ARG, "eta_k must be finite and > 0");
+    cudaStream_t s = (cudaStream_t)stream;
+    bool al = true;
+    int rc;
+    VecParams P;
+    base_params(ctx, P);
+    for (int i = 0; i < ctx->cfg.n; ++i) {
+        if ((rc = check_vector(ctx, grads[i], grad_elem_size(ctx->cfg.grad_dtype), "grads[i]", &al)) != INTSGD_OK) return rc;
+        if ((rc = check_vector(ctx, h_local[i], 4, "h_local[i]", &al)) != INTSGD_OK) return rc;
+        P.in[i] = grads[i];
+        P.out[i] = h_local[i];
+    }
+    if ((rc = check_vector(ctx, h_global, 4, "h_global", &al)) != INTSGD_OK) return rc;
+    if ((rc = check_vector(ctx, x, 4, "x", &al)) != INTSGD_OK) return rc;
+    if (agg && (rc = check_vector(ctx, agg, 4, "agg", &al)) != INTSGD_OK) return rc;
+    P.h = h_global;
+    P.x = x;
+    P.agg = agg;
+    ctx->last_stream = s;
+    if ((rc = launch_scale(ctx, eta_k, -1.0, s)) != INTSGD_OK) return rc;
+    return launch_diana(ctx, P, al, s);
 }
 
 int intsgd_step_host(intsgd_ctx* ctx, const void* const* host_grads, float* host_x, int32_t* host_agg,

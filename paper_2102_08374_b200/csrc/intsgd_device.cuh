@@ -30,7 +30,9 @@ struct DevState {
     int32_t max_abs_agg;
     uint32_t ticket;   // blocks that have published their partial in the running reduction
     int32_t fault;     // sticky: a bounded wait inside a kernel gave up (results of that step are invalid)
-    int32_t pad;
+    float ainv;        // fp32(1 / alpha)        } factors of the IntDIANA step (Algorithm 3),
+    float cn;          // fp32(1 / (n alpha))    } written by the scale kernel with alpha and c
+    float eta32;       // fp32(eta)              }
 };
 
 // Philox4x32-10 round keys (key schedule done once on the host: the key is the same for every
@@ -59,6 +61,7 @@ struct VecParams {
     float* x;
     int32_t* agg;
     const float* x_prev;                  // sqdiff only
+    float* h;                             // IntDIANA: global shift (out[i] holds the local shifts)
     DevState* st;
     double* partials;                     // one slot per block of the grid
     int64_t d;

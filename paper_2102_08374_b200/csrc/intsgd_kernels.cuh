@@ -36,6 +36,9 @@ __global__ void scale_kernel(DevState* st, double sqrt_d, double two_n, double n
     st->r = r;
     st->alpha = alpha;
     st->c = c;
+    st->ainv = __double2float_rn(__ddiv_rn(1.0, (double)alpha));
+    st->cn = __double2float_rn(__ddiv_rn(1.0, __dmul_rn(n_as_double, (double)alpha)));
+    st->eta32 = __double2float_rn(eta);
     st->status = INTSGD_OK;
 }
 
