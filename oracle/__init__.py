@@ -86,6 +86,8 @@ def lib() -> C.CDLL:
                                             C.c_int, C.c_uint64, C.c_uint32, C.POINTER(C.c_void_p), C.c_void_p,
                                             C.c_void_p, C.c_void_p, f64p, u64p, u64p, u64p, i32p]
         L.orc_diana_step_window.restype = None
+        L.orc_heuristic_scale.argtypes = [C.c_float, C.c_int32, C.c_int32, C.c_double, i32p, f32p, f32p]
+        L.orc_heuristic_scale.restype = C.c_int
     return _lib
 
 
@@ -394,3 +396,20 @@ class OracleIntDIANA:
         self.step += 1
         out.update(r=r, alpha64=a64, alpha=a32)
         return out
+
+
+def heuristic_scale(grads, n, nb, eta):
+    """Heuristic IntSGD scale (Section 5.2): profiling pass for the largest |g| over all workers (NaN
+    ignored), then alpha = (2^nb - 1) / (n 2^max_exp).  Returns (max_abs, max_exp, alpha32, c32) or
+    None when no scale exists (all zero, or an infinite entry)."""
+    biggest = np.float32(0.0)
+    for g in grads:
+        g = np.ascontiguousarray(g)
+        g32 = (g.astype(np.uint32) << 16).view(np.float32) if g.dtype == np.uint16 else g
+        m = np.fmax.reduce(np.abs(g32), initial=np.float32(0.0))     # fmax ignores NaN
+        biggest = np.fmax(biggest, m)
+    e, a, c = C.c_int32(), C.c_float(), C.c_float()
+    rc = lib().orc_heuristic_scale(float(biggest), n, nb, float(eta), C.byref(e), C.byref(a), C.byref(c))
+    if rc != 0:
+        return None
+    return float(biggest), e.value, np.float32(a.value), np.float32(c.value)

@@ -351,4 +351,24 @@ void orc_diana_step_window(const void* const* grads, int grad_dtype, int32_t n, 
     *dx2_out = dx2;
 }
 
+// ---- Heuristic IntSGD (Section 5.2, the SwitchML rule the paper compares against) ---------------
+// alpha = (2^nb - 1) / (n 2^max_exp), where max_exp is the exponent of the largest absolute value
+// in the package rounded up: the smallest integer e with max|g| <= 2^e.  Then |alpha g| <=
+// (2^nb - 1) / n for every entry.  c = eta / (n alpha) as in Algorithm 1.  Returns 0, or -1 when
+// max_abs is zero, negative or not finite (no scale exists).
+int orc_heuristic_scale(float max_abs, int32_t n, int32_t nb, double eta, int32_t* max_exp_out, float* alpha_out,
+                        float* c_out) {
+    if (!(max_abs > 0.0f) || !std::isfinite(max_abs)) return -1;
+    int e = 0;
+    const float m = std::frexp(max_abs, &e);   // max_abs = m 2^e, m in [0.5, 1)
+    const int max_exp = (m == 0.5f) ? e - 1 : e;
+    const double levels = std::ldexp(1.0, nb) - 1.0;
+    const double alpha64 = levels / ((double)n * std::ldexp(1.0, max_exp));
+    const float alpha = (float)alpha64;
+    *max_exp_out = max_exp;
+    *alpha_out = alpha;
+    *c_out = (float)(eta / ((double)n * (double)alpha));
+    return 0;
+}
+
 }  // extern "C"
