@@ -160,6 +160,17 @@ int intsgd_step(intsgd_ctx* ctx, const void* const* grads, void* const* payload_
 int intsgd_diana_step(intsgd_ctx* ctx, const void* const* grads, float* const* h_local, float* h_global, float* x,
                       int32_t* agg, double eta_k, void* stream);
 
+/* One step of Heuristic IntSGD (Section 5.2 of the paper: the SwitchML scale the paper compares with,
+ * built to show what its profiling pass costs).  A first pass over all n gradients finds max |g|
+ * (NaN ignored); alpha = (2^num_bits - 1) / (n 2^max_exp), max_exp the smallest integer with
+ * max |g| <= 2^max_exp, so that n |alpha g| <= 2^num_bits - 1; then the fused kernel of intsgd_step
+ * runs with that alpha and c = eta_k / (n alpha).  The moving average r is left untouched; dx2,
+ * counters and the step index are updated as usual.  If max |g| is zero or infinite the step is not
+ * applied (INTSGD_ERR_SCALE_NONFINITE at intsgd_get_stats).  Values beyond the context's clip limit
+ * still clip (num_bits = 32 exceeds the default int32 limit by a factor of two). */
+int intsgd_heuristic_step(intsgd_ctx* ctx, const void* const* grads, float* x, int32_t* agg, double eta_k,
+                          int32_t num_bits, void* stream);
+
 /* The same step for a caller whose buffers are in HOST memory (pinned memory recommended):
  * copies the n gradients and x to device staging buffers owned by the context (allocated on
  * first use: n*d gradient values + d floats + d int32), runs intsgd_step, copies x (and agg if

@@ -34,7 +34,7 @@ EXPORTS = [
     "intsgd_aggregate", "intsgd_step", "intsgd_step_host", "intsgd_get_stats", "intsgd_get_state",
     "intsgd_set_state", "intsgd_set_launch", "intsgd_set_fused_path", "intsgd_launch_count", "intsgd_last_error",
     "intsgd_sqdiff_noalloc", "intsgd_set_blocks", "intsgd_get_block_state", "intsgd_set_block_state",
-    "intsgd_diana_step",
+    "intsgd_diana_step", "intsgd_heuristic_step",
 ]
 
 
@@ -86,6 +86,7 @@ def load() -> C.CDLL:
     lib.intsgd_aggregate.argtypes = [vp, C.POINTER(vp), vp, vp, vp]
     lib.intsgd_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, vp, f64, i32, vp]
     lib.intsgd_diana_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, vp, vp, f64, vp]
+    lib.intsgd_heuristic_step.argtypes = [vp, C.POINTER(vp), vp, vp, f64, i32, vp]
     lib.intsgd_step_host.argtypes = [vp, C.POINTER(vp), vp, vp, f64, i32, vp]
     lib.intsgd_get_stats.argtypes = [vp, C.POINTER(Stats)]
     lib.intsgd_get_state.argtypes = [vp, C.POINTER(State)]
@@ -203,6 +204,10 @@ class IntSGD:
     def intsgd_diana_step(self, grads, h_local, h_global, x, agg=None, *, eta_k, stream=None):
         self._check(self._lib.intsgd_diana_step(self._ctx, _ptr_array(grads), _ptr_array(h_local), _addr(h_global),
                                                 _addr(x), _addr(agg), eta_k, stream))
+
+    def intsgd_heuristic_step(self, grads, x, agg=None, *, eta_k, num_bits, stream=None):
+        self._check(self._lib.intsgd_heuristic_step(self._ctx, _ptr_array(grads), _addr(x), _addr(agg), eta_k,
+                                                    num_bits, stream))
 
     def intsgd_step_host(self, host_grads, host_x, host_agg=None, *, eta_k, mode=MODE_FUSED, stream=None):
         self._check(self._lib.intsgd_step_host(self._ctx, _ptr_array(host_grads), _addr(host_x),

@@ -694,6 +694,45 @@ int intsgd_diana_step(intsgd_ctx* ctx, const void* const* grads, float* const* h
     return launch_diana(ctx, P, al, s);
 }
 
+int intsgd_heuristic_step(intsgd_ctx* ctx, const void* const* grads, float* x, int32_t* agg, double eta_k,
+                          int32_t num_bits, void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (ctx->bs.B > 0) return block_mode_unsupported(ctx, "intsgd_heuristic_step");
+    if (!grads) return fail(ctx, INTSGD_ERR_INVALID_ARG, "grads is NULL");
+    if (num_bits < 2 || num_bits > 32) return fail(ctx, INTSGD_ERR_INVALID_ARG, "num_bits must be in 2..32");
+    if (!(eta_k > 0.0) || !std::isfinite(eta_k)) return fail(ctx, INTSGD_ERR_INVALID_ARG, "eta_k must be finite and > 0");
+    cudaStream_t s = (cudaStream_t)stream;
+    bool al = true;
+    int rc;
+    VecParams P;
+    base_params(ctx, P);
+    for (int i = 0; i < ctx->cfg.n; ++i) {
+        if ((rc = check_vector(ctx, grads[i], grad_elem_size(ctx->cfg.grad_dtype), "grads[i]", &al)) != INTSGD_OK) return rc;
+        P.in[i] = grads[i];
+    }
+    if ((rc = check_vector(ctx, x, 4, "x", &al)) != INTSGD_OK) return rc;
+    if (agg && (rc = check_vector(ctx, agg, 4, "agg", &al)) != INTSGD_OK) return rc;
+    P.x = x;
+    P.agg = agg;
+    ctx->last_stream = s;
+    // profiling pass over every worker's gradient
+    const int n = ctx->cfg.n;
+    dim3 grid((unsigned)grid_for(ctx, (ctx->cfg.d + 3) / 4), (unsigned)n, 1);
+    int per = (ctx->sm_count * ctx->blocks_per_sm + n - 1) / n;
+    if (per < 1) per = 1;
+    if ((int)grid.x > per) grid.x = (unsigned)per;
+    const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
+    if (!bf16 && al) maxabs_kernel<INTSGD_GRAD_F32, true><<<grid, ctx->threads, 0, s>>>(P);
+    else if (!bf16) maxabs_kernel<INTSGD_GRAD_F32, false><<<grid, ctx->threads, 0, s>>>(P);
+    else if (al) maxabs_kernel<INTSGD_GRAD_BF16, true><<<grid, ctx->threads, 0, s>>>(P);
+    else maxabs_kernel<INTSGD_GRAD_BF16, false><<<grid, ctx->threads, 0, s>>>(P);
+    if ((rc = after_launch(ctx, "maxabs_kernel")) != INTSGD_OK) return rc;
+    heuristic_scale_kernel<<<1, 32, 0, s>>>(ctx->d_state, (double)n, eta_k, std::ldexp(1.0, num_bits) - 1.0, n);
+    if ((rc = after_launch(ctx, "heuristic_scale_kernel")) != INTSGD_OK) return rc;
+    return launch_fused(ctx, P, al, s);
+}
+
 int intsgd_step_host(intsgd_ctx* ctx, const void* const* host_grads, float* host_x, int32_t* host_agg,
                      double eta_k, int32_t mode, void* stream) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;

@@ -33,6 +33,8 @@ struct DevState {
     float ainv;        // fp32(1 / alpha)        } factors of the IntDIANA step (Algorithm 3),
     float cn;          // fp32(1 / (n alpha))    } written by the scale kernel with alpha and c
     float eta32;       // fp32(eta)              }
+    uint32_t maxabs_bits;   // heuristic scale: bits of max |g| found by the profiling pass (0 between steps)
+    uint32_t pad2;
 };
 
 // Philox4x32-10 round keys (key schedule done once on the host: the key is the same for every

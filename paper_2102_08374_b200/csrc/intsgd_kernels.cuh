@@ -313,4 +313,58 @@ __global__ void __launch_bounds__(kMaxThreads) sqdiff_kernel(const __grid_consta
     grid_finalize(acc, P.st, P.partials, false);
 }
 
+// ----------------------------------------------------------------------------------------
+// Heuristic IntSGD (Section 5.2 of the paper, the SwitchML rule): a profiling pass finds the largest
+// |g| over all workers (NaN ignored), then alpha = (2^nb - 1) / (n 2^max_exp) with max_exp the
+// smallest integer e such that max|g| <= 2^e.  grid = (blocks, workers).
+// ----------------------------------------------------------------------------------------
+template <int GRAD, bool ALIGNED>
+__global__ void __launch_bounds__(kMaxThreads) maxabs_kernel(const __grid_constant__ VecParams P) {
+    const void* g = P.in[blockIdx.y];
+    float m = 0.0f;
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
+        const float4 v = load_grad4<GRAD, ALIGNED>(g, unit);
+        m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        for (int64_t j = full << 2; j < P.d; ++j) m = fmaxf(m, fabsf(grad_at<GRAD>(g, j)));
+    // non-negative, NaN-free floats order like their bit patterns
+    const unsigned bits = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(m));
+    if ((threadIdx.x & 31) == 0 && bits) atomicMax(&P.st->maxabs_bits, bits);
+}
+
+__global__ void heuristic_scale_kernel(DevState* st, double n_as_double, double eta, double levels, int32_t n) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const float max_abs = __uint_as_float(st->maxabs_bits);
+    st->maxabs_bits = 0;
+    for (int i = 0; i < n; ++i) st->clip_count[i] = 0;
+    st->nonfinite = 0;
+    st->agg_overflow = 0;
+    st->max_abs_agg = 0;
+    st->ticket = 0;
+    if (!(max_abs > 0.0f) || !(max_abs <= 3.402823466e+38f)) {
+        st->status = INTSGD_ERR_SCALE_NONFINITE;
+        return;
+    }
+    int e = 0;
+    const float mant = frexpf(max_abs, &e);
+    const int max_exp = (mant == 0.5f) ? e - 1 : e;
+    const double alpha64 = __ddiv_rn(levels, __dmul_rn(n_as_double, ldexp(1.0, max_exp)));
+    const float alpha = __double2float_rn(alpha64);
+    const float c = __double2float_rn(__ddiv_rn(eta, __dmul_rn(n_as_double, (double)alpha)));
+    const bool ok = (alpha > 0.0f) && (alpha <= 3.402823466e+38f) && (c > 0.0f) && (c <= 3.402823466e+38f);
+    if (!ok) {
+        st->status = INTSGD_ERR_SCALE_NONFINITE;
+        return;
+    }
+    st->alpha = alpha;
+    st->c = c;
+    st->ainv = __double2float_rn(__ddiv_rn(1.0, (double)alpha));
+    st->cn = __double2float_rn(__ddiv_rn(1.0, __dmul_rn(n_as_double, (double)alpha)));
+    st->eta32 = __double2float_rn(eta);
+    st->status = INTSGD_OK;
+}
+
 }  // namespace intsgd
