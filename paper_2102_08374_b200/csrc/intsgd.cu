@@ -730,7 +730,14 @@ int intsgd_heuristic_step(intsgd_ctx* ctx, const void* const* grads, float* x, i
     if ((rc = after_launch(ctx, "maxabs_kernel")) != INTSGD_OK) return rc;
     heuristic_scale_kernel<<<1, 32, 0, s>>>(ctx->d_state, (double)n, eta_k, std::ldexp(1.0, num_bits) - 1.0, n);
     if ((rc = after_launch(ctx, "heuristic_scale_kernel")) != INTSGD_OK) return rc;
-    return launch_fused(ctx, P, al, s);
+    // The pipelined kernel sums integer-valued floats and is exact only below 2^24 / n per value; this
+    // rule fills num_bits on purpose, so wide settings run the direct kernel (int32 accumulation).
+    const double top = (std::ldexp(1.0, num_bits) - 1.0) / (double)n;
+    const int saved_path = ctx->fused_path;
+    if (top > (double)((1 << 24) / n - 2)) ctx->fused_path = 1;
+    rc = launch_fused(ctx, P, al, s);
+    ctx->fused_path = saved_path;
+    return rc;
 }
 
 int intsgd_step_host(intsgd_ctx* ctx, const void* const* host_grads, float* host_x, int32_t* host_agg,
