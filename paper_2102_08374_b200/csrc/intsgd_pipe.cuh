@@ -250,6 +250,8 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         const uint32_t step = st->step;
         const BlockParams& bp = P.bp;
         uint32_t s = 0, phase = 0;
+        float max_sum = 0.0f;                                            // max |S| over fast-path units
+        const bool count_overflow = P.agg_limit != 0x7FFFFFFF;          // int8 wire: count |S| > 127
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             const int64_t unit0 = tile * kTileUnits + c;
             float4 xo[UPT];
@@ -353,22 +355,40 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 }
                 if (!active[k]) continue;
                 int4 S;
+                float2 S01, S23;   // the sums as floats (exact on the fast path)
                 if (ua[k].m <= PP.fast_limit) {
-                    S = make_int4(__float2int_rn(ua[k].F01.x), __float2int_rn(ua[k].F01.y),
-                                  __float2int_rn(ua[k].F23.x), __float2int_rn(ua[k].F23.y));
+                    S01 = ua[k].F01;
+                    S23 = ua[k].F23;
+                    S = make_int4(__float2int_rn(S01.x), __float2int_rn(S01.y), __float2int_rn(S23.x), __float2int_rn(S23.y));
+                    max_sum = absmax3_nan(max_sum, S01.x, S01.y);
+                    max_sum = absmax3_nan(max_sum, S23.x, S23.y);
+                    if (count_overflow)
+                        acc.overflow += (fabsf(S01.x) > 127.0f) + (fabsf(S01.y) > 127.0f) + (fabsf(S23.x) > 127.0f) +
+                                        (fabsf(S23.y) > 127.0f);
                 } else {
                     S = redo_unit<GRAD, ROUND>(P, unit, make_float4(alpha, alpha, alpha, alpha), step, s_cnt);
+                    S01 = make_float2(__int2float_rn(S.x), __int2float_rn(S.y));
+                    S23 = make_float2(__int2float_rn(S.z), __int2float_rn(S.w));
+                    note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
+                    note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
                 }
-                float4 xn;
-                xn.x = update_coord(xo[k].x, S.x, cdec, acc.dx2);
-                xn.y = update_coord(xo[k].y, S.y, cdec, acc.dx2);
-                xn.z = update_coord(xo[k].z, S.z, cdec, acc.dx2);
-                xn.w = update_coord(xo[k].w, S.w, cdec, acc.dx2);
-                store_f4<true>(P.x, unit, xn);
+                // t = fl(c S); x_new = fl(x - t); dj = fl(x_new - x): packed, each rounded once
+                const float2 neg1 = make_float2(-1.0f, -1.0f), c2 = make_float2(cdec, cdec);
+                const float2 xo01 = make_float2(xo[k].x, xo[k].y), xo23 = make_float2(xo[k].z, xo[k].w);
+                const float2 xn01 = __ffma2_rn(__fmul2_rn(c2, S01), neg1, xo01);
+                const float2 xn23 = __ffma2_rn(__fmul2_rn(c2, S23), neg1, xo23);
+                const float2 d01 = __ffma2_rn(xo01, neg1, xn01), d23 = __ffma2_rn(xo23, neg1, xn23);
+                acc.dx2 = __fma_rn((double)d01.x, (double)d01.x, acc.dx2);
+                acc.dx2 = __fma_rn((double)d01.y, (double)d01.y, acc.dx2);
+                acc.dx2 = __fma_rn((double)d23.x, (double)d23.x, acc.dx2);
+                acc.dx2 = __fma_rn((double)d23.y, (double)d23.y, acc.dx2);
+                store_f4<true>(P.x, unit, make_float4(xn01.x, xn01.y, xn23.x, xn23.y));
                 if (P.agg) store_i4<true>(P.agg, unit, S);
-                note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
-                note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
             }
+        }
+        {   // fold the float-tracked maximum of the fast-path sums (integers below 2^24) into the counters
+            const int mf = __float2int_rn(max_sum);
+            acc.max_abs = acc.max_abs > mf ? acc.max_abs : mf;
         }
         if (!ok) atomicExch(&s_fault, 1);
 
