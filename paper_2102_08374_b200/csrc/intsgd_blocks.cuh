@@ -224,8 +224,8 @@ __global__ void __launch_bounds__(128) block_norm_kernel(DevState* st, BlockStat
 // iteration (one chunk); the loop condition is warp-uniform so that every lane reaches the shuffles.
 // ---------------------------------------------------------------------------------------------
 template <int ROUND>
-__device__ __forceinline__ int4 round_unit_scaled(float4 g, float2 a01, float2 a23, uint4 w, float Lf, u64* clip_slot,
-                                                  u64* nonfinite_slot) {
+__device__ __forceinline__ int4 round_unit_scaled(float4 g, float2 a01, float2 a23, uint4 w, float Lf, cnt_t* clip_slot,
+                                                  cnt_t* nonfinite_slot) {
     const float y0 = __fmul_rn(a01.x, g.x), y1 = __fmul_rn(a01.y, g.y);
     const float y2 = __fmul_rn(a23.x, g.z), y3 = __fmul_rn(a23.y, g.w);
     const bool in_range = (fabsf(y0) <= Lf) & (fabsf(y1) <= Lf) & (fabsf(y2) <= Lf) & (fabsf(y3) <= Lf);
@@ -236,10 +236,7 @@ __device__ __forceinline__ int4 round_unit_scaled(float4 g, float2 a01, float2 a
         q.z = round_in_range<ROUND>(y2, w.z);
         q.w = round_in_range<ROUND>(y3, w.w);
     } else {
-        q.x = round_checked<ROUND>(y0, w.x, Lf, clip_slot, nonfinite_slot);
-        q.y = round_checked<ROUND>(y1, w.y, Lf, clip_slot, nonfinite_slot);
-        q.z = round_checked<ROUND>(y2, w.z, Lf, clip_slot, nonfinite_slot);
-        q.w = round_checked<ROUND>(y3, w.w, Lf, clip_slot, nonfinite_slot);
+        q = round_unit_checked<ROUND>(y0, y1, y2, y3, w, Lf, clip_slot, nonfinite_slot);
     }
     return q;
 }
@@ -253,7 +250,7 @@ __device__ __forceinline__ void coord_scale(const BlockParams& bp, int64_t j, fl
 
 template <int GRAD, bool ALIGNED, int ROUND>
 __global__ void __launch_bounds__(512) fused_step_blocks_kernel(const __grid_constant__ VecParams P) {
-    __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
+    __shared__ cnt_t s_cnt[INTSGD_MAX_WORKERS + 1];
     DevState* st = P.st;
     if (st->status != INTSGD_OK) return;
     counters_init(s_cnt);
@@ -261,7 +258,7 @@ __global__ void __launch_bounds__(512) fused_step_blocks_kernel(const __grid_con
     const uint32_t step = st->step;
     const int n = P.n;
     const int lane = threadIdx.x & 31;
-    u64* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
+    cnt_t* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
     ThreadAcc acc = {0.0, 0, 0u};
 
     const int64_t full = P.d >> 2;   // == bp.covered_end / 4

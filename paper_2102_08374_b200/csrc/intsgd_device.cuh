@@ -13,6 +13,9 @@
 namespace intsgd {
 
 typedef unsigned long long u64;
+// Per-block event counters in shared memory: 32 bits are enough (a block cannot see 2^32 elements of
+// one worker within the memory of one GPU) and 32-bit shared-memory atomics are native.
+typedef uint32_t cnt_t;
 
 // ----------------------------------------------------------------------------------------
 // Device-resident state.  The first 32 bytes have the layout of intsgd_state.
@@ -177,20 +180,44 @@ __device__ __forceinline__ int round_in_range(float y, uint32_t w) {
 // Full rule with clipping: values outside [-Lf, Lf] saturate, NaN becomes 0, and the event is
 // counted (Section 5.1: local values are clipped so that the aggregate fits the wire type).
 template <int ROUND>
-__device__ __noinline__ int round_checked(float y, uint32_t w, float Lf, u64* clip_slot, u64* nonfinite_slot) {
+__device__ __forceinline__ int round_full(float y, uint32_t w, float Lf, uint32_t& clipped, uint32_t& nonfinite) {
     if (fabsf(y) <= Lf) return round_in_range<ROUND>(y, w);
-    atomicAdd(clip_slot, 1ull);
-    if (!(fabsf(y) <= 3.402823466e+38f)) atomicAdd(nonfinite_slot, 1ull);   // NaN or +-Inf
+    clipped += 1;
+    if (!(fabsf(y) <= 3.402823466e+38f)) nonfinite += 1;   // NaN or +-Inf
     if (y > Lf) return (int)Lf;
     if (y < -Lf) return -(int)Lf;
     return 0;   // NaN
 }
 
+template <int ROUND>
+__device__ __noinline__ int round_checked(float y, uint32_t w, float Lf, cnt_t* clip_slot, cnt_t* nonfinite_slot) {
+    uint32_t clipped = 0, nonfinite = 0;
+    const int q = round_full<ROUND>(y, w, Lf, clipped, nonfinite);
+    if (clipped) atomicAdd(clip_slot, clipped);
+    if (nonfinite) atomicAdd(nonfinite_slot, nonfinite);
+    return q;
+}
+
+// Four values of one worker with the full rule; the counters get one atomic per unit at most.
+template <int ROUND>
+__device__ __noinline__ int4 round_unit_checked(float y0, float y1, float y2, float y3, uint4 w, float Lf,
+                                                cnt_t* clip_slot, cnt_t* nonfinite_slot) {
+    uint32_t clipped = 0, nonfinite = 0;
+    int4 q;
+    q.x = round_full<ROUND>(y0, w.x, Lf, clipped, nonfinite);
+    q.y = round_full<ROUND>(y1, w.y, Lf, clipped, nonfinite);
+    q.z = round_full<ROUND>(y2, w.z, Lf, clipped, nonfinite);
+    q.w = round_full<ROUND>(y3, w.w, Lf, clipped, nonfinite);
+    if (clipped) atomicAdd(clip_slot, clipped);
+    if (nonfinite) atomicAdd(nonfinite_slot, nonfinite);
+    return q;
+}
+
 // One unit of one worker: scale, round, clip.  The common case (all four values in range) has no
 // clamp and no counter traffic.
 template <int ROUND>
-__device__ __forceinline__ int4 round_unit(float4 g, float alpha, uint4 w, float Lf, u64* clip_slot,
-                                           u64* nonfinite_slot) {
+__device__ __forceinline__ int4 round_unit(float4 g, float alpha, uint4 w, float Lf, cnt_t* clip_slot,
+                                           cnt_t* nonfinite_slot) {
     const float y0 = __fmul_rn(alpha, g.x), y1 = __fmul_rn(alpha, g.y);
     const float y2 = __fmul_rn(alpha, g.z), y3 = __fmul_rn(alpha, g.w);
     const bool in_range = (fabsf(y0) <= Lf) & (fabsf(y1) <= Lf) & (fabsf(y2) <= Lf) & (fabsf(y3) <= Lf);
@@ -201,10 +228,7 @@ __device__ __forceinline__ int4 round_unit(float4 g, float alpha, uint4 w, float
         q.z = round_in_range<ROUND>(y2, w.z);
         q.w = round_in_range<ROUND>(y3, w.w);
     } else {
-        q.x = round_checked<ROUND>(y0, w.x, Lf, clip_slot, nonfinite_slot);
-        q.y = round_checked<ROUND>(y1, w.y, Lf, clip_slot, nonfinite_slot);
-        q.z = round_checked<ROUND>(y2, w.z, Lf, clip_slot, nonfinite_slot);
-        q.w = round_checked<ROUND>(y3, w.w, Lf, clip_slot, nonfinite_slot);
+        q = round_unit_checked<ROUND>(y0, y1, y2, y3, w, Lf, clip_slot, nonfinite_slot);
     }
     return q;
 }
@@ -295,11 +319,11 @@ __device__ __forceinline__ void grid_finalize(const ThreadAcc& a, DevState* st, 
 
 // Per-block clip / non-finite counters live in shared memory (slot i < n: worker i's clipped
 // count, slot INTSGD_MAX_WORKERS: non-finite count) and are flushed once per block.
-__device__ __forceinline__ void counters_init(u64* s_cnt) {
+__device__ __forceinline__ void counters_init(cnt_t* s_cnt) {
     for (int t = threadIdx.x; t <= INTSGD_MAX_WORKERS; t += blockDim.x) s_cnt[t] = 0;
     __syncthreads();
 }
-__device__ __forceinline__ void counters_flush(const u64* s_cnt, DevState* st) {
+__device__ __forceinline__ void counters_flush(const cnt_t* s_cnt, DevState* st) {
     __syncthreads();
     for (int t = threadIdx.x; t <= INTSGD_MAX_WORKERS; t += blockDim.x) {
         const u64 v = s_cnt[t];

@@ -29,7 +29,7 @@ __device__ __forceinline__ float diana_coord(float x_old, float h_old, int S, co
 
 template <int ROUND>
 __device__ __forceinline__ int diana_worker_coord(float g, float& h, uint32_t w, const DianaFactors& f, float Lf,
-                                                  u64* clip_slot, u64* nonf_slot) {
+                                                  cnt_t* clip_slot, cnt_t* nonf_slot) {
     const float y = __fmul_rn(f.alpha, __fsub_rn(g, h));
     const int q = (fabsf(y) <= Lf) ? round_in_range<ROUND>(y, w) : round_checked<ROUND>(y, w, Lf, clip_slot, nonf_slot);
     h = __fadd_rn(h, __fmul_rn(f.ainv, __int2float_rn(q)));
@@ -39,14 +39,14 @@ __device__ __forceinline__ int diana_worker_coord(float g, float& h, uint32_t w,
 // Direct (grid-stride) kernel: one unit of 4 coordinates per thread and iteration.
 template <int GRAD, bool ALIGNED, int ROUND>
 __global__ void __launch_bounds__(512) diana_step_kernel(const __grid_constant__ VecParams P) {
-    __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
+    __shared__ cnt_t s_cnt[INTSGD_MAX_WORKERS + 1];
     DevState* st = P.st;
     if (st->status != INTSGD_OK) return;
     counters_init(s_cnt);
     const DianaFactors f = {st->alpha, st->ainv, st->cn, st->eta32};
     const uint32_t step = st->step;
     const int n = P.n;
-    u64* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
+    cnt_t* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
     ThreadAcc acc = {0.0, 0, 0u};
 
     const int64_t full = P.d >> 2;

@@ -65,7 +65,7 @@ __device__ __forceinline__ void store_payload4(void* base, int64_t unit, int4 q,
 
 template <int GRAD, int PAY, bool ALIGNED, int ROUND>
 __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_constant__ VecParams P) {
-    __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
+    __shared__ cnt_t s_cnt[INTSGD_MAX_WORKERS + 1];
     DevState* st = P.st;
     if (st->status != INTSGD_OK) return;
     counters_init(s_cnt);
@@ -75,8 +75,8 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
     const uint32_t worker = (uint32_t)(P.worker_base + slot);
     const void* g = P.in[slot];
     void* out = P.out[slot];
-    u64* clip_slot = &s_cnt[worker];
-    u64* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
+    cnt_t* clip_slot = &s_cnt[worker];
+    cnt_t* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
 
     const int64_t full = P.d >> 2;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -201,14 +201,14 @@ __global__ void __launch_bounds__(kMaxThreads) aggregate_kernel(const __grid_con
 // ----------------------------------------------------------------------------------------
 template <int GRAD, bool ALIGNED, int ROUND>
 __global__ void __launch_bounds__(kMaxThreads) fused_step_kernel(const __grid_constant__ VecParams P) {
-    __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
+    __shared__ cnt_t s_cnt[INTSGD_MAX_WORKERS + 1];
     DevState* st = P.st;
     if (st->status != INTSGD_OK) return;
     counters_init(s_cnt);
     const float alpha = st->alpha, c = st->c;
     const uint32_t step = st->step;
     const int n = P.n;
-    u64* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
+    cnt_t* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
     ThreadAcc acc = {0.0, 0, 0u};
 
     const int64_t full = P.d >> 2;

@@ -108,19 +108,20 @@ __device__ __forceinline__ void consume_unit(float4 g, float2 alpha01, float2 al
 // Exact redo of one unit from global memory with the full clipping rule and the counters (rare:
 // some |alpha g| outside the fast range, or a NaN/Inf).  The fast path has counted nothing.
 template <int GRAD, int ROUND>
-__device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float4 alpha4, uint32_t step, u64* s_cnt) {
+__device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float4 alpha4, uint32_t step, cnt_t* s_cnt) {
     const float av[4] = {alpha4.x, alpha4.y, alpha4.z, alpha4.w};
     int S[4] = {0, 0, 0, 0};
     for (int i = 0; i < P.n; ++i) {
         const float4 g = load_grad4<GRAD, true>(P.in[i], unit);
         uint4 w = make_uint4(0, 0, 0, 0);
         if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, (uint32_t)i, step, P.keys);
-        const float gv[4] = {g.x, g.y, g.z, g.w};
-        const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
-        for (int e = 0; e < 4; ++e) {
-            const float y = __fmul_rn(av[e], gv[e]);
-            S[e] += round_checked<ROUND>(y, wv[e], P.Lf, &s_cnt[i], &s_cnt[INTSGD_MAX_WORKERS]);
-        }
+        uint32_t clipped = 0, nonfinite = 0;
+        S[0] += round_full<ROUND>(__fmul_rn(av[0], g.x), w.x, P.Lf, clipped, nonfinite);
+        S[1] += round_full<ROUND>(__fmul_rn(av[1], g.y), w.y, P.Lf, clipped, nonfinite);
+        S[2] += round_full<ROUND>(__fmul_rn(av[2], g.z), w.z, P.Lf, clipped, nonfinite);
+        S[3] += round_full<ROUND>(__fmul_rn(av[3], g.w), w.w, P.Lf, clipped, nonfinite);
+        if (clipped) atomicAdd(&s_cnt[i], clipped);
+        if (nonfinite) atomicAdd(&s_cnt[INTSGD_MAX_WORKERS], nonfinite);
     }
     return make_int4(S[0], S[1], S[2], S[3]);
 }
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(16) uint4 s_tab[INTSGD_MAX_WORKERS];
     __shared__ uint64_t full_bar[NS], empty_bar[NS];
-    __shared__ u64 s_cnt[INTSGD_MAX_WORKERS + 1];
+    __shared__ cnt_t s_cnt[INTSGD_MAX_WORKERS + 1];
     __shared__ int s_fault;
 
     const VecParams& P = PP.v;
