@@ -29,6 +29,32 @@ METRIC = "fused IntSGD step throughput"
 UNIT = "gradient elements/s"
 HBM_FALLBACK_GBS = 6650.0
 
+# DRAM traffic of the fused kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum;
+# command and figures in profiles/fused_pipe_kernel_d24_n16_ncu_full.md): bytes per coordinate of the
+# captured case (d = 2^24, n = 16, fp32, int32 aggregate), valid for the kernel sources with this hash.
+# Any change to the kernel sources makes `roofline.traffic` null until the counters are taken again.
+NCU_TRAFFIC = {"sources_sha256": "bb6be72ac34aa26293852d713466a102b4a50ba2b933515ee1620b4cd32ea8cf",
+               "bytes_per_coordinate": 1.266304e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
+
+
+def kernel_sources_hash():
+    import hashlib
+    h = hashlib.sha256()
+    for f in sorted((ROOT / "paper_2102_08374_b200" / "csrc").glob("*")):
+        h.update(f.name.encode())
+        h.update(f.read_bytes())
+    return h.hexdigest()
+
+
+def traffic_per_launch(args, d):
+    """Measured DRAM bytes per launch, scaled to d (traffic is proportional to d), or None."""
+    t = NCU_TRAFFIC
+    same = (args.workers == t["workers"] and args.grad == t["grad"] and args.mode == t["mode"]
+            and args.rounding == "random")
+    if not same or kernel_sources_hash() != t["sources_sha256"]:
+        return None
+    return t["bytes_per_coordinate"] * d
+
 
 def parse_args():
     p = argparse.ArgumentParser()
@@ -263,7 +289,7 @@ def main():
     peak, peak_kind = measured_hbm_peak()
     achieved = bytes_per_launch / (avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
+                "traffic": traffic_per_launch(args, d), "peak_source": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
                 "algorithmic_bytes_per_launch": bytes_per_launch, "kernel_ms_avg": avg_ms,
                 "kernel_ms_median": statistics.median(per_step_ms),
                 "note": "per-step CUDA-event time (one-thread scale kernel + the vector kernel(s))"}
