@@ -39,55 +39,59 @@ def build(force: bool = False) -> Path:
 _lib = None
 
 
+def _declare(L: C.CDLL) -> C.CDLL:
+    """Attach argument and result types to the oracle's entry points."""
+    u32p, f32p, i32p = C.POINTER(C.c_uint32), C.POINTER(C.c_float), C.POINTER(C.c_int32)
+    f64p, u64p = C.POINTER(C.c_double), C.POINTER(C.c_uint64)
+    L.orc_philox4x32_10.argtypes = [u32p, u32p, u32p]
+    L.orc_philox4x32_10.restype = None
+    L.orc_draw_word.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64]
+    L.orc_draw_word.restype = C.c_uint32
+    L.orc_uniform_from_word.argtypes = [C.c_uint32]
+    L.orc_uniform_from_word.restype = C.c_float
+    L.orc_int_round.argtypes = [C.c_float, C.c_float]
+    L.orc_int_round.restype = C.c_int32
+    L.orc_int_round_nearest.argtypes = [C.c_float]
+    L.orc_int_round_nearest.restype = C.c_int32
+    L.orc_limit_as_float.argtypes = [C.c_int64]
+    L.orc_limit_as_float.restype = C.c_float
+    L.orc_scale.argtypes = [C.c_int64, C.c_int32, C.c_double, C.c_double, C.c_double,
+                            C.c_double, C.c_double, f64p, f64p, f32p, f32p]
+    L.orc_scale.restype = None
+    L.orc_scale_block.argtypes = [C.c_int64, C.c_int64, C.c_int32, C.c_double, C.c_double,
+                                  C.c_double, C.c_double, C.c_double, f64p, f64p, f32p, f32p]
+    L.orc_scale_block.restype = None
+    L.orc_encode.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_float, C.c_int64,
+                             C.c_int, C.c_int, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
+                             C.c_void_p, u64p, u64p]
+    L.orc_encode.restype = None
+    L.orc_aggregate.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64,
+                                C.c_float, C.c_void_p, C.c_void_p, f64p, u64p, i32p]
+    L.orc_aggregate.restype = None
+    L.orc_exact_step.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64,
+                                 C.c_double, C.c_void_p, f64p]
+    L.orc_exact_step.restype = None
+    L.orc_sqdiff.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
+    L.orc_sqdiff.restype = C.c_double
+    L.orc_step_window.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64,
+                                  C.c_int64, C.c_float, C.c_float, C.c_int64, C.c_int, C.c_int,
+                                  C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                  f64p, u64p, u64p, u64p, i32p]
+    L.orc_step_window.restype = None
+    L.orc_diana_step_window.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64, C.c_int64,
+                                        C.c_float, C.c_float, C.c_float, C.c_float, C.c_int64, C.c_int,
+                                        C.c_int, C.c_uint64, C.c_uint32, C.POINTER(C.c_void_p), C.c_void_p,
+                                        C.c_void_p, C.c_void_p, f64p, u64p, u64p, u64p, i32p]
+    L.orc_diana_step_window.restype = None
+    L.orc_heuristic_scale.argtypes = [C.c_float, C.c_int32, C.c_int32, C.c_double, i32p, f32p, f32p]
+    L.orc_heuristic_scale.restype = C.c_int
+    return L
+
+
 def lib() -> C.CDLL:
     global _lib
     if _lib is None:
-        _lib = C.CDLL(str(build()))
-        L = _lib
-        u32p, f32p, i32p = C.POINTER(C.c_uint32), C.POINTER(C.c_float), C.POINTER(C.c_int32)
-        f64p, u64p = C.POINTER(C.c_double), C.POINTER(C.c_uint64)
-        L.orc_philox4x32_10.argtypes = [u32p, u32p, u32p]
-        L.orc_philox4x32_10.restype = None
-        L.orc_draw_word.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64]
-        L.orc_draw_word.restype = C.c_uint32
-        L.orc_uniform_from_word.argtypes = [C.c_uint32]
-        L.orc_uniform_from_word.restype = C.c_float
-        L.orc_int_round.argtypes = [C.c_float, C.c_float]
-        L.orc_int_round.restype = C.c_int32
-        L.orc_int_round_nearest.argtypes = [C.c_float]
-        L.orc_int_round_nearest.restype = C.c_int32
-        L.orc_limit_as_float.argtypes = [C.c_int64]
-        L.orc_limit_as_float.restype = C.c_float
-        L.orc_scale.argtypes = [C.c_int64, C.c_int32, C.c_double, C.c_double, C.c_double,
-                                C.c_double, C.c_double, f64p, f64p, f32p, f32p]
-        L.orc_scale.restype = None
-        L.orc_scale_block.argtypes = [C.c_int64, C.c_int64, C.c_int32, C.c_double, C.c_double,
-                                      C.c_double, C.c_double, C.c_double, f64p, f64p, f32p, f32p]
-        L.orc_scale_block.restype = None
-        L.orc_encode.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_float, C.c_int64,
-                                 C.c_int, C.c_int, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
-                                 C.c_void_p, u64p, u64p]
-        L.orc_encode.restype = None
-        L.orc_aggregate.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64,
-                                    C.c_float, C.c_void_p, C.c_void_p, f64p, u64p, i32p]
-        L.orc_aggregate.restype = None
-        L.orc_exact_step.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64,
-                                     C.c_double, C.c_void_p, f64p]
-        L.orc_exact_step.restype = None
-        L.orc_sqdiff.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
-        L.orc_sqdiff.restype = C.c_double
-        L.orc_step_window.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64,
-                                      C.c_int64, C.c_float, C.c_float, C.c_int64, C.c_int, C.c_int,
-                                      C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
-                                      f64p, u64p, u64p, u64p, i32p]
-        L.orc_step_window.restype = None
-        L.orc_diana_step_window.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int64, C.c_int64,
-                                            C.c_float, C.c_float, C.c_float, C.c_float, C.c_int64, C.c_int,
-                                            C.c_int, C.c_uint64, C.c_uint32, C.POINTER(C.c_void_p), C.c_void_p,
-                                            C.c_void_p, C.c_void_p, f64p, u64p, u64p, u64p, i32p]
-        L.orc_diana_step_window.restype = None
-        L.orc_heuristic_scale.argtypes = [C.c_float, C.c_int32, C.c_int32, C.c_double, i32p, f32p, f32p]
-        L.orc_heuristic_scale.restype = C.c_int
+        _lib = _declare(C.CDLL(str(build())))
     return _lib
 
 

@@ -151,3 +151,12 @@ def test_default_int32_limit_makes_the_sum_fit():
         Lf = oracle.limit_as_float(L)
         assert clip == 2 and q[0] == int(Lf) and q[1] == -int(Lf) and q[2] == 1
         assert n * int(Lf) <= 2**31 - 1
+
+
+def test_non_finite_values_on_the_int32_wire():
+    # NaN -> 0, +-Inf -> +-Lf, each counted as clipped and as non-finite
+    n = 4
+    Lf = int(oracle.limit_as_float(oracle.default_clip_limit(n, PAYLOAD_I32)))
+    g = np.array([np.nan, np.inf, -np.inf, 1.0, -np.nan], dtype=np.float32)
+    q, clip, nonf = oracle.encode(g, np.float32(1.0), worker=0, step=0, seed=0, n=n)
+    assert list(q) == [0, Lf, -Lf, 1, 0] and clip == 4 and nonf == 4
