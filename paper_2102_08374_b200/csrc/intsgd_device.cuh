@@ -162,6 +162,20 @@ __device__ __forceinline__ int4 load_i4(const int32_t* base, int64_t unit) {
     return make_int4(__ldcs(p), __ldcs(p + 1), __ldcs(p + 2), __ldcs(p + 3));
 }
 
+// max(|a|, |b|, |c|), NaN if any input is NaN (three-input max of sm_100).
+__device__ __forceinline__ float absmax3_nan(float a, float b, float c) {
+    float d;
+    asm("max.NaN.abs.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// 1.0f if a < b else 0.0f, in one instruction.
+__device__ __forceinline__ float lt_as_float(float a, float b) {
+    float d;
+    asm("set.lt.f32.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
 // ----------------------------------------------------------------------------------------
 // Rounding.  y = fl32(alpha * g).  Random: f = floor(y), p = fl32(y - f),
 // u = (w >> 8) * 2^-24, q = f + [u < p]  (Int(t), Section 2 of the paper).
@@ -213,24 +227,36 @@ __device__ __noinline__ int4 round_unit_checked(float y0, float y1, float y2, fl
     return q;
 }
 
+// Four in-range values at once with packed fp32x2 arithmetic; bit-identical to round_in_range on
+// each (the same separately rounded steps: floor, y - f, scaling by 2^24, compare, add).
+template <int ROUND>
+__device__ __forceinline__ int4 round4_in_range(float2 y01, float2 y23, uint4 w) {
+    if (ROUND == INTSGD_ROUND_NEAREST)
+        return make_int4(__float2int_rn(y01.x), __float2int_rn(y01.y), __float2int_rn(y23.x), __float2int_rn(y23.y));
+    const float2 f01 = make_float2(floorf(y01.x), floorf(y01.y));
+    const float2 f23 = make_float2(floorf(y23.x), floorf(y23.y));
+    const float2 neg1 = make_float2(-1.0f, -1.0f), scale = make_float2(16777216.0f, 16777216.0f);
+    const float2 p01 = __fmul2_rn(__ffma2_rn(f01, neg1, y01), scale);
+    const float2 p23 = __fmul2_rn(__ffma2_rn(f23, neg1, y23), scale);
+    const float2 u01 = make_float2(lt_as_float(__uint2float_rn(w.x >> 8), p01.x),
+                                   lt_as_float(__uint2float_rn(w.y >> 8), p01.y));
+    const float2 u23 = make_float2(lt_as_float(__uint2float_rn(w.z >> 8), p23.x),
+                                   lt_as_float(__uint2float_rn(w.w >> 8), p23.y));
+    const float2 q01 = __fadd2_rn(f01, u01), q23 = __fadd2_rn(f23, u23);
+    return make_int4(__float2int_rz(q01.x), __float2int_rz(q01.y), __float2int_rz(q23.x), __float2int_rz(q23.y));
+}
+
 // One unit of one worker: scale, round, clip.  The common case (all four values in range) has no
 // clamp and no counter traffic.
 template <int ROUND>
 __device__ __forceinline__ int4 round_unit(float4 g, float alpha, uint4 w, float Lf, cnt_t* clip_slot,
                                            cnt_t* nonfinite_slot) {
-    const float y0 = __fmul_rn(alpha, g.x), y1 = __fmul_rn(alpha, g.y);
-    const float y2 = __fmul_rn(alpha, g.z), y3 = __fmul_rn(alpha, g.w);
-    const bool in_range = (fabsf(y0) <= Lf) & (fabsf(y1) <= Lf) & (fabsf(y2) <= Lf) & (fabsf(y3) <= Lf);
-    int4 q;
-    if (in_range) {
-        q.x = round_in_range<ROUND>(y0, w.x);
-        q.y = round_in_range<ROUND>(y1, w.y);
-        q.z = round_in_range<ROUND>(y2, w.z);
-        q.w = round_in_range<ROUND>(y3, w.w);
-    } else {
-        q = round_unit_checked<ROUND>(y0, y1, y2, y3, w, Lf, clip_slot, nonfinite_slot);
-    }
-    return q;
+    const float2 alpha2 = make_float2(alpha, alpha);
+    const float2 y01 = __fmul2_rn(alpha2, make_float2(g.x, g.y));
+    const float2 y23 = __fmul2_rn(alpha2, make_float2(g.z, g.w));
+    const float m = absmax3_nan(absmax3_nan(y01.x, y01.y, y23.x), y23.y, y23.y);
+    if (m <= Lf) return round4_in_range<ROUND>(y01, y23, w);   // false for NaN
+    return round_unit_checked<ROUND>(y01.x, y01.y, y23.x, y23.y, w, Lf, clip_slot, nonfinite_slot);
 }
 
 // Decode + update of one coordinate: t = fl32(c * float(S)); x_new = fl32(x - t); the squared

@@ -53,8 +53,8 @@ __device__ __forceinline__ void store_payload4(void* base, int64_t unit, int4 q,
         __stcs(p, q.x); __stcs(p + 1, q.y); __stcs(p + 2, q.z); __stcs(p + 3, q.w);
     } else {
         if (aligned) {
-            const uint32_t packed = (uint32_t)(q.x & 0xFF) | ((uint32_t)(q.y & 0xFF) << 8) |
-                                    ((uint32_t)(q.z & 0xFF) << 16) | ((uint32_t)(q.w & 0xFF) << 24);
+            // low bytes of the four values, in order
+            const uint32_t packed = __byte_perm(__byte_perm(q.x, q.y, 0x0040), __byte_perm(q.z, q.w, 0x0040), 0x5410);
             __stcs((uint32_t*)base + unit, packed);
             return;
         }

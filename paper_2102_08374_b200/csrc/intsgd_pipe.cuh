@@ -57,20 +57,6 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
                  : "memory");
 }
 
-// max(|a|, |b|, |c|), NaN if any input is NaN (three-input max of sm_100).
-__device__ __forceinline__ float absmax3_nan(float a, float b, float c) {
-    float d;
-    asm("max.NaN.abs.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-
-// 1.0f if a < b else 0.0f, in one instruction.
-__device__ __forceinline__ float lt_as_float(float a, float b) {
-    float d;
-    asm("set.lt.f32.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
-    return d;
-}
-
 // ---- per-unit arithmetic ------------------------------------------------------------------------
 // Fast path of one worker's unit.  Floors and up-decisions are accumulated as integer-valued
 // floats (exact: the host caps the fast-path magnitude T so that n * (T + 1) <= 2^24, and T never
