@@ -80,12 +80,34 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
 
     const int64_t full = P.d >> 2;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
-        const float4 gv = load_grad4<GRAD, ALIGNED>(g, unit);
-        uint4 w = make_uint4(0, 0, 0, 0);
-        if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, worker, step, P.keys);
-        const int4 q = round_unit<ROUND>(gv, alpha, w, P.Lf, clip_slot, nonf_slot);
-        store_payload4<PAY>(out, unit, q, ALIGNED);
+    if (PAY == INTSGD_PAYLOAD_I32) {
+        // 8 bytes per element: bound by memory, so keep the register count (and occupancy) of the plain loop
+        for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
+            const float4 gv = load_grad4<GRAD, ALIGNED>(g, unit);
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, worker, step, P.keys);
+            store_payload4<PAY>(out, unit, round_unit<ROUND>(gv, alpha, w, P.Lf, clip_slot, nonf_slot), ALIGNED);
+        }
+    } else {
+        // 5 (3) bytes per element: bound by arithmetic.  Two units per iteration, and the next pair's
+        // loads issued before this pair is rounded, so two Philox chains overlap and cover the latency.
+        int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        float4 ga = make_float4(0.f, 0.f, 0.f, 0.f), gb = ga;
+        if (unit < full) ga = load_grad4<GRAD, ALIGNED>(g, unit);
+        if (unit + stride < full) gb = load_grad4<GRAD, ALIGNED>(g, unit + stride);
+        for (; unit < full; unit += 2 * stride) {
+            const int64_t ub = unit + stride, na = unit + 2 * stride, nb = unit + 3 * stride;
+            const float4 ca = ga, cb = gb;
+            if (na < full) ga = load_grad4<GRAD, ALIGNED>(g, na);
+            if (nb < full) gb = load_grad4<GRAD, ALIGNED>(g, nb);
+            uint4 wa = make_uint4(0, 0, 0, 0), wb = wa;
+            if (ROUND == INTSGD_ROUND_RANDOM) {
+                wa = draw_unit(unit, worker, step, P.keys);
+                wb = draw_unit(ub, worker, step, P.keys);
+            }
+            store_payload4<PAY>(out, unit, round_unit<ROUND>(ca, alpha, wa, P.Lf, clip_slot, nonf_slot), ALIGNED);
+            if (ub < full) store_payload4<PAY>(out, ub, round_unit<ROUND>(cb, alpha, wb, P.Lf, clip_slot, nonf_slot), ALIGNED);
+        }
     }
     const int tail = (int)(P.d & 3);
     if (tail && blockIdx.x == 0 && threadIdx.x == 0) {
