@@ -21,7 +21,7 @@ _LIB = _HERE / "liboracle_intsgd.so"
 
 GRAD_F32, GRAD_BF16 = 0, 1
 PAYLOAD_I32, PAYLOAD_I8 = 0, 1
-ROUND_RANDOM, ROUND_NEAREST = 0, 1
+ROUND_RANDOM, ROUND_NEAREST, ROUND_RANDOM16 = 0, 1, 2
 INT32_MAX = 2**31 - 1
 
 
@@ -49,6 +49,8 @@ def _declare(L: C.CDLL) -> C.CDLL:
     L.orc_draw_word.restype = C.c_uint32
     L.orc_uniform_from_word.argtypes = [C.c_uint32]
     L.orc_uniform_from_word.restype = C.c_float
+    L.orc_draw_uniform16.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64]
+    L.orc_draw_uniform16.restype = C.c_float
     L.orc_int_round.argtypes = [C.c_float, C.c_float]
     L.orc_int_round.restype = C.c_int32
     L.orc_int_round_nearest.argtypes = [C.c_float]
@@ -127,6 +129,10 @@ def philox4x32_10(ctr, key) -> tuple[int, int, int, int]:
 
 def draw_word(seed: int, step: int, worker: int, j: int) -> int:
     return int(lib().orc_draw_word(seed, step, worker, j))
+
+
+def draw_uniform16(seed: int, step: int, worker: int, j: int) -> float:
+    return float(lib().orc_draw_uniform16(seed, step, worker, j))
 
 
 def uniform_from_word(w: int) -> float:

@@ -72,6 +72,25 @@ uint32_t draw_word(uint64_t seed, uint32_t step, uint32_t worker, uint64_t j) {
     return out[j & 3];
 }
 
+// Optional coarser stream ("16-bit draws", rounding mode 2): one Philox block serves 8 coordinates.
+// Unit u = j / 4 is paired with the unit 512 places away: pair index P = ((u >> 10) << 9) | (u & 511),
+// half h = (u >> 9) & 1; the block of counter (P low, P high, worker, step) gives words 2h and 2h + 1
+// to the unit, and coordinate e = j mod 4 takes the low (e even) or high (e odd) 16 bits of word
+// 2h + e / 2.  The uniform is that value times 2^-16.
+float draw_uniform16(uint64_t seed, uint32_t step, uint32_t worker, uint64_t j) {
+    const uint64_t u = j >> 2;
+    const uint32_t e = (uint32_t)(j & 3);
+    const uint64_t pair = ((u >> 10) << 9) | (u & 511);
+    const uint32_t h = (uint32_t)((u >> 9) & 1);
+    const uint32_t ctr[4] = {(uint32_t)pair, (uint32_t)(pair >> 32), worker, step};
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t out[4];
+    philox4x32_10(ctr, key, out);
+    const uint32_t word = out[2 * h + (e >> 1)];
+    const uint32_t v = (e & 1) ? (word >> 16) : (word & 0xFFFFu);
+    return (float)v * 1.52587890625e-5f;  // 2^-16
+}
+
 // 24-bit uniform in [0, 1): the top 24 bits of the word times 2^-24; exact in fp32.
 float uniform_from_word(uint32_t w) {
     return (float)(w >> 8) * 5.9604644775390625e-8f;  // 2^-24
@@ -139,6 +158,9 @@ uint32_t orc_draw_word(uint64_t seed, uint32_t step, uint32_t worker, uint64_t j
     return draw_word(seed, step, worker, j);
 }
 float orc_uniform_from_word(uint32_t w) { return uniform_from_word(w); }
+float orc_draw_uniform16(uint64_t seed, uint32_t step, uint32_t worker, uint64_t j) {
+    return draw_uniform16(seed, step, worker, j);
+}
 
 // ---- Int(t), Section 2 ------------------------------------------------------------------
 int32_t orc_int_round(float y, float u) { return (int32_t)int_round_random(y, u); }
@@ -192,7 +214,8 @@ void orc_scale_block(int64_t d, int64_t d_l, int32_t n, double eta, double beta,
 // ---- Algorithm 1, "scale and round the local gradient": Int(alpha_k g_i) ----------------
 // One worker, coordinates [j0, j0 + count) of a vector whose element 0 is grad[0]
 // (grad, payload and u_inject are indexed relative to j0; the random stream by j0 + t).
-// grad_dtype 0 = fp32, 1 = bf16; payload_dtype 0 = int32, 1 = int8; rounding 0 = random,
+// grad_dtype 0 = fp32, 1 = bf16; payload_dtype 0 = int32, 1 = int8; rounding 0 = random (24-bit draws),
+// 2 = random with the 16-bit draws of draw_uniform16,
 // 1 = nearest-even.  u_inject (nullable) replaces the Philox draw, for hand examples.
 void orc_encode(const void* grad, int grad_dtype, int64_t j0, int64_t count, float alpha,
                 int64_t L, int payload_dtype, int rounding, uint64_t seed, uint32_t step,
@@ -203,9 +226,10 @@ void orc_encode(const void* grad, int grad_dtype, int64_t j0, int64_t count, flo
         const float g = load_grad(grad, grad_dtype, t);
         const float y = alpha * g;
         float u = 0.0f;
-        if (rounding == 0) {
-            u = u_inject ? u_inject[t]
-                         : uniform_from_word(draw_word(seed, step, worker, (uint64_t)(j0 + t)));
+        if (rounding != 1) {
+            if (u_inject) u = u_inject[t];
+            else if (rounding == 2) u = draw_uniform16(seed, step, worker, (uint64_t)(j0 + t));
+            else u = uniform_from_word(draw_word(seed, step, worker, (uint64_t)(j0 + t)));
         }
         const Rounded r = round_and_clip(y, u, Lf, rounding);
         if (r.clipped) *clip_count += 1;
@@ -326,7 +350,8 @@ void orc_diana_step_window(const void* const* grads, int grad_dtype, int32_t n, 
             const float v = g - h_local[i][t];
             const float y = alpha * v;
             float u = 0.0f;
-            if (rounding == 0) u = uniform_from_word(draw_word(seed, step, (uint32_t)i, (uint64_t)(j0 + t)));
+            if (rounding == 2) u = draw_uniform16(seed, step, (uint32_t)i, (uint64_t)(j0 + t));
+            else if (rounding == 0) u = uniform_from_word(draw_word(seed, step, (uint32_t)i, (uint64_t)(j0 + t)));
             const Rounded r = round_and_clip(y, u, Lf, rounding);
             if (r.clipped) clip_count[i] += 1;
             if (r.nonfinite) *nonfinite_count += 1;

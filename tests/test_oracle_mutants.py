@@ -9,6 +9,7 @@ import pytest
 import oracle
 import test_oracle_blocks as tb
 import test_oracle_diana as td
+import test_oracle_draw16 as t16
 import test_oracle_heuristic as th
 import test_oracle_philox as tp
 import test_oracle_rounding as tr
@@ -51,6 +52,9 @@ MUTANTS = [
     ("sqdiff: difference not squared", "s += (double)dj * (double)dj;", "s += (double)dj;"),
     ("diana: shift moved by the raw integer", "const float dq = ainv * (float)r.q;", "const float dq = (float)r.q;"),
     ("diana: estimator without the shift", "const float gt = h_global[t] + dec;", "const float gt = dec;"),
+    ("16-bit draws: halves swapped", "const uint32_t v = (e & 1) ? (word >> 16) : (word & 0xFFFFu);", "const uint32_t v = (e & 1) ? (word & 0xFFFFu) : (word >> 16);"),
+    ("16-bit draws: wrong word of the pair", "const uint32_t word = out[2 * h + (e >> 1)];", "const uint32_t word = out[h + (e >> 1)];"),
+    ("16-bit draws: partner at distance 256", "const uint32_t h = (uint32_t)((u >> 9) & 1);", "const uint32_t h = (uint32_t)((u >> 8) & 1);"),
     ("heuristic: exponent rounded down", "const int max_exp = (m == 0.5f) ? e - 1 : e;", "const int max_exp = e - 1;"),
 ]
 
@@ -91,6 +95,7 @@ def _battery():
     td.test_hand_example(GOLDEN)
     td.test_zero_shifts_give_the_intsgd_integers_and_step()
     th.test_hand_values()
+    t16.test_layout_against_an_independent_statement()
 
 
 def test_the_unmodified_oracle_passes_the_battery(tmp_path, monkeypatch):
