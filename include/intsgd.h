@@ -59,6 +59,13 @@ extern "C" {
 #define INTSGD_PAYLOAD_I8    1
 #define INTSGD_ROUND_RANDOM  0   /* Int(t) of Section 2 */
 #define INTSGD_ROUND_NEAREST 1   /* "IntSGD (Determ.)" of Section 5.1: nearest, ties to even */
+#define INTSGD_ROUND_RANDOM16 2  /* Int(t) with 16-bit draws: one Philox block serves 8 coordinates.
+                                    Unit u = j / 4 shares the block of pair index
+                                    P = ((u >> 10) << 9) | (u & 511) (counter (P low, P high, worker, step))
+                                    with unit u ^ 512, takes words 2h and 2h + 1 (h = bit 9 of u); coordinate
+                                    e = j mod 4 uses the low (e even) or high (e odd) 16 bits v of word
+                                    2h + e / 2; rounds up iff v * 2^-16 < fl32(y - floor(y)).  Bias at most
+                                    2^-16 per value.  Halves the random-number work: an option, not the default */
 #define INTSGD_MODE_EXACT      0 /* Algorithm 1, Init line: x <- x - eta (1/n) sum_i g_i, uncompressed */
 #define INTSGD_MODE_TWO_KERNEL 1 /* encode every worker to a payload buffer, then aggregate */
 #define INTSGD_MODE_FUSED      2 /* one pass, payloads never reach memory */

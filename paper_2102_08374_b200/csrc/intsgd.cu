@@ -175,6 +175,8 @@ template <int GRAD, int PAY, bool ALIGNED>
 void launch_encode_r(const intsgd_ctx* ctx, const VecParams& P, dim3 grid, cudaStream_t s) {
     if (ctx->cfg.rounding == INTSGD_ROUND_NEAREST)
         encode_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
+    else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM16)
+        encode_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_RANDOM16><<<grid, ctx->threads, 0, s>>>(P);
     else
         encode_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
@@ -214,6 +216,8 @@ template <int GRAD, bool ALIGNED>
 void launch_fused_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStream_t s) {
     if (ctx->cfg.rounding == INTSGD_ROUND_NEAREST)
         fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
+    else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM16)
+        fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM16><<<grid, ctx->threads, 0, s>>>(P);
     else
         fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
@@ -292,11 +296,13 @@ int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     // Floors and up-decisions are summed as integer-valued floats: exact while n * (T + 1) <= 2^24.
     const float t_max = (float)((1 << 24) / ctx->cfg.n - 2);
     PP.fast_limit = ctx->Lf < t_max ? ctx->Lf : t_max;
-    const bool nearest = ctx->cfg.rounding == INTSGD_ROUND_NEAREST;
+    const int rounding = ctx->cfg.rounding;
     cudaError_t e;
-    if (!bf16 && !nearest) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_RANDOM>(ctx, PP, s);
+    if (!bf16 && rounding == INTSGD_ROUND_RANDOM) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_RANDOM>(ctx, PP, s);
+    else if (!bf16 && rounding == INTSGD_ROUND_RANDOM16) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_RANDOM16>(ctx, PP, s);
     else if (!bf16) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_NEAREST>(ctx, PP, s);
-    else if (!nearest) e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_RANDOM>(ctx, PP, s);
+    else if (rounding == INTSGD_ROUND_RANDOM) e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_RANDOM>(ctx, PP, s);
+    else if (rounding == INTSGD_ROUND_RANDOM16) e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_RANDOM16>(ctx, PP, s);
     else e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_NEAREST>(ctx, PP, s);
     if (e != cudaSuccess) {
         std::snprintf(ctx->err, 256, "fused_pipe_kernel setup failed: %s", cudaGetErrorString(e));
@@ -311,6 +317,8 @@ template <int GRAD, bool ALIGNED>
 void launch_fused_blocks_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStream_t s) {
     if (ctx->cfg.rounding == INTSGD_ROUND_NEAREST)
         fused_step_blocks_kernel<GRAD, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
+    else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM16)
+        fused_step_blocks_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM16><<<grid, ctx->threads, 0, s>>>(P);
     else
         fused_step_blocks_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
@@ -343,6 +351,8 @@ template <int GRAD, bool ALIGNED>
 void launch_diana_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStream_t s) {
     if (ctx->cfg.rounding == INTSGD_ROUND_NEAREST)
         diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
+    else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM16)
+        diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM16><<<grid, ctx->threads, 0, s>>>(P);
     else
         diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
@@ -474,7 +484,8 @@ int intsgd_create(intsgd_ctx** out, const intsgd_config* cfg) {
         return fail(nullptr, INTSGD_ERR_INVALID_ARG, "bad grad_dtype");
     if (cfg->payload_dtype != INTSGD_PAYLOAD_I32 && cfg->payload_dtype != INTSGD_PAYLOAD_I8)
         return fail(nullptr, INTSGD_ERR_INVALID_ARG, "bad payload_dtype");
-    if (cfg->rounding != INTSGD_ROUND_RANDOM && cfg->rounding != INTSGD_ROUND_NEAREST)
+    if (cfg->rounding != INTSGD_ROUND_RANDOM && cfg->rounding != INTSGD_ROUND_NEAREST &&
+        cfg->rounding != INTSGD_ROUND_RANDOM16)
         return fail(nullptr, INTSGD_ERR_INVALID_ARG, "bad rounding");
     if (!(cfg->beta >= 0.0 && cfg->beta < 1.0)) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "beta must be in [0, 1)");
     if (!(cfg->eps >= 0.0) || !std::isfinite(cfg->eps)) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "eps must be finite and >= 0");

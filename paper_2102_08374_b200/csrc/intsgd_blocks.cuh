@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(512) fused_step_blocks_kernel(const __grid_con
             for (int i = 0; i < n; ++i) {
                 const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
                 uint4 w = make_uint4(0, 0, 0, 0);
-                if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, (uint32_t)i, step, P.keys);
+                if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, (uint32_t)i, step, P.keys);
                 const int4 q = round_unit_scaled<ROUND>(gv, us.a01, us.a23, w, P.Lf, &s_cnt[i], nonf_slot);
                 S.x += q.x; S.y += q.y; S.z += q.z; S.w += q.w;
             }
@@ -303,8 +303,8 @@ __global__ void __launch_bounds__(512) fused_step_blocks_kernel(const __grid_con
             int S = 0;
             for (int i = 0; i < n; ++i) {
                 uint32_t word = 0;
-                if (ROUND == INTSGD_ROUND_RANDOM) {
-                    const uint4 w4 = draw_unit(j >> 2, (uint32_t)i, step, P.keys);
+                if (ROUND != INTSGD_ROUND_NEAREST) {
+                    const uint4 w4 = draw_unit<ROUND>(j >> 2, (uint32_t)i, step, P.keys);
                     const uint32_t wv[4] = {w4.x, w4.y, w4.z, w4.w};
                     word = wv[j & 3];
                 }

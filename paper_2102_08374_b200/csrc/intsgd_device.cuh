@@ -101,10 +101,32 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
-// Random words of unit `unit` (coordinates 4*unit .. 4*unit+3) of `worker` at `step`.
-__device__ __forceinline__ uint4 draw_unit(int64_t unit, uint32_t worker, uint32_t step,
-                                           const PhiloxKeys& K) {
+// Random draws of unit `unit` (coordinates 4*unit .. 4*unit+3) of `worker` at `step`, one per
+// coordinate.  Default stream: the four words of Philox block `unit`; the rounding uses their top 24
+// bits.  INTSGD_ROUND_RANDOM16: 16-bit draws; unit u shares the block of pair index
+// P = ((u >> 10) << 9) | (u & 511) with the unit 512 places away, takes words 2h and 2h + 1
+// (h = bit 9 of u), and coordinate e gets the low (e even) or high (e odd) half of word 2h + e / 2.
+template <int ROUND>
+__device__ __forceinline__ uint4 draw_unit(int64_t unit, uint32_t worker, uint32_t step, const PhiloxKeys& K) {
+    if (ROUND == INTSGD_ROUND_RANDOM16) {
+        const uint64_t u = (uint64_t)unit;
+        const uint64_t pair = ((u >> 10) << 9) | (u & 511);
+        const uint4 w = philox4x32_10((uint32_t)pair, (uint32_t)(pair >> 32), worker, step, K);
+        const bool h = (u >> 9) & 1;
+        const uint32_t a = h ? w.z : w.x, b = h ? w.w : w.y;
+        return make_uint4(a & 0xFFFFu, a >> 16, b & 0xFFFFu, b >> 16);
+    }
     return philox4x32_10((uint32_t)unit, (uint32_t)((uint64_t)unit >> 32), worker, step, K);
+}
+
+// The draw as a float and the power of two that scales the fractional part to the same range.
+template <int ROUND>
+__device__ __forceinline__ float draw_as_float(uint32_t w) {
+    return (ROUND == INTSGD_ROUND_RANDOM16) ? __uint2float_rn(w) : __uint2float_rn(w >> 8);
+}
+template <int ROUND>
+__device__ __forceinline__ float draw_scale() {
+    return (ROUND == INTSGD_ROUND_RANDOM16) ? 65536.0f : 16777216.0f;
 }
 
 // ----------------------------------------------------------------------------------------
@@ -180,14 +202,15 @@ __device__ __forceinline__ float lt_as_float(float a, float b) {
 // Rounding.  y = fl32(alpha * g).  Random: f = floor(y), p = fl32(y - f),
 // u = (w >> 8) * 2^-24, q = f + [u < p]  (Int(t), Section 2 of the paper).
 // The comparison is done as (float)(w >> 8) < p * 2^24: both scalings are exact.
+// (With 16-bit draws: (float)v < p * 2^16.)
 // ----------------------------------------------------------------------------------------
 template <int ROUND>
 __device__ __forceinline__ int round_in_range(float y, uint32_t w) {
     if (ROUND == INTSGD_ROUND_NEAREST) return __float2int_rn(y);
     const float f = floorf(y);
     const float p = __fsub_rn(y, f);
-    const float uf = __uint2float_rn(w >> 8);
-    const float pscaled = __fmul_rn(p, 16777216.0f);
+    const float uf = draw_as_float<ROUND>(w);
+    const float pscaled = __fmul_rn(p, draw_scale<ROUND>());
     return __float2int_rz(f) + (uf < pscaled ? 1 : 0);
 }
 
@@ -235,13 +258,11 @@ __device__ __forceinline__ int4 round4_in_range(float2 y01, float2 y23, uint4 w)
         return make_int4(__float2int_rn(y01.x), __float2int_rn(y01.y), __float2int_rn(y23.x), __float2int_rn(y23.y));
     const float2 f01 = make_float2(floorf(y01.x), floorf(y01.y));
     const float2 f23 = make_float2(floorf(y23.x), floorf(y23.y));
-    const float2 neg1 = make_float2(-1.0f, -1.0f), scale = make_float2(16777216.0f, 16777216.0f);
+    const float2 neg1 = make_float2(-1.0f, -1.0f), scale = make_float2(draw_scale<ROUND>(), draw_scale<ROUND>());
     const float2 p01 = __fmul2_rn(__ffma2_rn(f01, neg1, y01), scale);
     const float2 p23 = __fmul2_rn(__ffma2_rn(f23, neg1, y23), scale);
-    const float2 u01 = make_float2(lt_as_float(__uint2float_rn(w.x >> 8), p01.x),
-                                   lt_as_float(__uint2float_rn(w.y >> 8), p01.y));
-    const float2 u23 = make_float2(lt_as_float(__uint2float_rn(w.z >> 8), p23.x),
-                                   lt_as_float(__uint2float_rn(w.w >> 8), p23.y));
+    const float2 u01 = make_float2(lt_as_float(draw_as_float<ROUND>(w.x), p01.x), lt_as_float(draw_as_float<ROUND>(w.y), p01.y));
+    const float2 u23 = make_float2(lt_as_float(draw_as_float<ROUND>(w.z), p23.x), lt_as_float(draw_as_float<ROUND>(w.w), p23.y));
     const float2 q01 = __fadd2_rn(f01, u01), q23 = __fadd2_rn(f23, u23);
     return make_int4(__float2int_rz(q01.x), __float2int_rz(q01.y), __float2int_rz(q23.x), __float2int_rz(q23.y));
 }

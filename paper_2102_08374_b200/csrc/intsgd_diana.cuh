@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(512) diana_step_kernel(const __grid_constant__
             float* hl = (float*)P.out[i];
             float4 hv = load_f4<ALIGNED>(hl, unit);
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, (uint32_t)i, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, (uint32_t)i, step, P.keys);
             S.x += diana_worker_coord<ROUND>(gv.x, hv.x, w.x, f, P.Lf, &s_cnt[i], nonf_slot);
             S.y += diana_worker_coord<ROUND>(gv.y, hv.y, w.y, f, P.Lf, &s_cnt[i], nonf_slot);
             S.z += diana_worker_coord<ROUND>(gv.z, hv.z, w.z, f, P.Lf, &s_cnt[i], nonf_slot);
@@ -83,8 +83,8 @@ __global__ void __launch_bounds__(512) diana_step_kernel(const __grid_constant__
             int S = 0;
             for (int i = 0; i < n; ++i) {
                 uint32_t word = 0;
-                if (ROUND == INTSGD_ROUND_RANDOM) {
-                    const uint4 w4 = draw_unit(j >> 2, (uint32_t)i, step, P.keys);
+                if (ROUND != INTSGD_ROUND_NEAREST) {
+                    const uint4 w4 = draw_unit<ROUND>(j >> 2, (uint32_t)i, step, P.keys);
                     const uint32_t wv[4] = {w4.x, w4.y, w4.z, w4.w};
                     word = wv[j & 3];
                 }

@@ -85,8 +85,31 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
         for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
             const float4 gv = load_grad4<GRAD, ALIGNED>(g, unit);
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, worker, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, worker, step, P.keys);
             store_payload4<PAY>(out, unit, round_unit<ROUND>(gv, alpha, w, P.Lf, clip_slot, nonf_slot), ALIGNED);
+        }
+    } else if (ROUND == INTSGD_ROUND_RANDOM16) {
+        // 16-bit draws: iterate over pair indices; the pair's two units (512 apart) share one Philox block.
+        const int64_t pairs = ((full + 1023) >> 10) << 9;
+        int64_t pr = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        int64_t ua = ((pr >> 9) << 10) | (pr & 511);
+        float4 ga = make_float4(0.f, 0.f, 0.f, 0.f), gb = ga;
+        if (pr < pairs && ua < full) ga = load_grad4<GRAD, ALIGNED>(g, ua);
+        if (pr < pairs && ua + 512 < full) gb = load_grad4<GRAD, ALIGNED>(g, ua + 512);
+        for (; pr < pairs; pr += stride) {
+            const int64_t np = pr + stride, nu = ((np >> 9) << 10) | (np & 511);
+            const int64_t ca_unit = ua;
+            const float4 ca = ga, cb = gb;
+            if (np < pairs && nu < full) ga = load_grad4<GRAD, ALIGNED>(g, nu);
+            if (np < pairs && nu + 512 < full) gb = load_grad4<GRAD, ALIGNED>(g, nu + 512);
+            ua = nu;
+            const uint4 w = philox4x32_10((uint32_t)pr, (uint32_t)((uint64_t)pr >> 32), worker, step, P.keys);
+            const uint4 wa = make_uint4(w.x & 0xFFFFu, w.x >> 16, w.y & 0xFFFFu, w.y >> 16);
+            const uint4 wb = make_uint4(w.z & 0xFFFFu, w.z >> 16, w.w & 0xFFFFu, w.w >> 16);
+            if (ca_unit < full)
+                store_payload4<PAY>(out, ca_unit, round_unit<ROUND>(ca, alpha, wa, P.Lf, clip_slot, nonf_slot), ALIGNED);
+            if (ca_unit + 512 < full)
+                store_payload4<PAY>(out, ca_unit + 512, round_unit<ROUND>(cb, alpha, wb, P.Lf, clip_slot, nonf_slot), ALIGNED);
         }
     } else {
         // 5 (3) bytes per element: bound by arithmetic.  Two units per iteration, and the next pair's
@@ -101,9 +124,9 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
             if (na < full) ga = load_grad4<GRAD, ALIGNED>(g, na);
             if (nb < full) gb = load_grad4<GRAD, ALIGNED>(g, nb);
             uint4 wa = make_uint4(0, 0, 0, 0), wb = wa;
-            if (ROUND == INTSGD_ROUND_RANDOM) {
-                wa = draw_unit(unit, worker, step, P.keys);
-                wb = draw_unit(ub, worker, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST) {
+                wa = draw_unit<ROUND>(unit, worker, step, P.keys);
+                wb = draw_unit<ROUND>(ub, worker, step, P.keys);
             }
             store_payload4<PAY>(out, unit, round_unit<ROUND>(ca, alpha, wa, P.Lf, clip_slot, nonf_slot), ALIGNED);
             if (ub < full) store_payload4<PAY>(out, ub, round_unit<ROUND>(cb, alpha, wb, P.Lf, clip_slot, nonf_slot), ALIGNED);
@@ -112,7 +135,7 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
     const int tail = (int)(P.d & 3);
     if (tail && blockIdx.x == 0 && threadIdx.x == 0) {
         uint4 w = make_uint4(0, 0, 0, 0);
-        if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(full, worker, step, P.keys);
+        if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(full, worker, step, P.keys);
         const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
         for (int e = 0; e < tail; ++e) {
             const int64_t j = 4 * full + e;
@@ -241,7 +264,7 @@ __global__ void __launch_bounds__(kMaxThreads) fused_step_kernel(const __grid_co
         for (int i = 0; i < n; ++i) {
             const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, (uint32_t)i, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, (uint32_t)i, step, P.keys);
             const int4 q = round_unit<ROUND>(gv, alpha, w, P.Lf, &s_cnt[i], nonf_slot);
             S.x += q.x; S.y += q.y; S.z += q.z; S.w += q.w;
         }
@@ -252,7 +275,7 @@ __global__ void __launch_bounds__(kMaxThreads) fused_step_kernel(const __grid_co
         int S[4] = {0, 0, 0, 0};
         for (int i = 0; i < n; ++i) {
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(full, (uint32_t)i, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(full, (uint32_t)i, step, P.keys);
             const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
             for (int e = 0; e < tail; ++e) {
                 const float y = __fmul_rn(alpha, grad_at<GRAD>(P.in[i], 4 * full + e));

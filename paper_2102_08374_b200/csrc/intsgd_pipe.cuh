@@ -80,13 +80,11 @@ __device__ __forceinline__ void consume_unit(float4 g, float2 alpha01, float2 al
     }
     const float2 f01 = make_float2(floorf(y01.x), floorf(y01.y));
     const float2 f23 = make_float2(floorf(y23.x), floorf(y23.y));
-    const float2 neg1 = make_float2(-1.0f, -1.0f), scale = make_float2(16777216.0f, 16777216.0f);
-    const float2 p01 = __fmul2_rn(__ffma2_rn(f01, neg1, y01), scale);   // fl32(y - f) * 2^24, both exact steps
+    const float2 neg1 = make_float2(-1.0f, -1.0f), scale = make_float2(draw_scale<ROUND>(), draw_scale<ROUND>());
+    const float2 p01 = __fmul2_rn(__ffma2_rn(f01, neg1, y01), scale);   // fl32(y - f) * 2^24 (2^16), both exact steps
     const float2 p23 = __fmul2_rn(__ffma2_rn(f23, neg1, y23), scale);
-    const float2 u01 = make_float2(lt_as_float(__uint2float_rn(w.x >> 8), p01.x),
-                                   lt_as_float(__uint2float_rn(w.y >> 8), p01.y));
-    const float2 u23 = make_float2(lt_as_float(__uint2float_rn(w.z >> 8), p23.x),
-                                   lt_as_float(__uint2float_rn(w.w >> 8), p23.y));
+    const float2 u01 = make_float2(lt_as_float(draw_as_float<ROUND>(w.x), p01.x), lt_as_float(draw_as_float<ROUND>(w.y), p01.y));
+    const float2 u23 = make_float2(lt_as_float(draw_as_float<ROUND>(w.z), p23.x), lt_as_float(draw_as_float<ROUND>(w.w), p23.y));
     u.F01 = __fadd2_rn(__fadd2_rn(u.F01, f01), u01);
     u.F23 = __fadd2_rn(__fadd2_rn(u.F23, f23), u23);
 }
@@ -100,7 +98,7 @@ __device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float4 
     for (int i = 0; i < P.n; ++i) {
         const float4 g = load_grad4<GRAD, true>(P.in[i], unit);
         uint4 w = make_uint4(0, 0, 0, 0);
-        if (ROUND == INTSGD_ROUND_RANDOM) w = draw_unit(unit, (uint32_t)i, step, P.keys);
+        if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, (uint32_t)i, step, P.keys);
         uint32_t clipped = 0, nonfinite = 0;
         S[0] += round_full<ROUND>(__fmul_rn(av[0], g.x), w.x, P.Lf, clipped, nonfinite);
         S[1] += round_full<ROUND>(__fmul_rn(av[1], g.y), w.y, P.Lf, clipped, nonfinite);
@@ -159,6 +157,12 @@ __device__ __forceinline__ uint4 philox_finish(const PhiloxThreadPart& t, uint4 
     return make_uint4(c0, c1, c2, c3);
 }
 
+// 16-bit draws: pair index of a unit, and the four draws of its half of the pair's Philox block.
+__device__ __forceinline__ uint32_t pair_index(uint32_t unit_lo) { return ((unit_lo >> 10) << 9) | (unit_lo & 511u); }
+__device__ __forceinline__ uint4 split16(uint32_t a, uint32_t b) {
+    return make_uint4(a & 0xFFFFu, a >> 16, b & 0xFFFFu, b >> 16);
+}
+
 template <int GRAD>
 __device__ __forceinline__ float4 lds_unit(const unsigned char* tile, int c) {
     if (GRAD == INTSGD_GRAD_F32) return *reinterpret_cast<const float4*>(tile + 16 * c);
@@ -175,6 +179,9 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
     constexpr int kUnitBytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
     constexpr int kTileUnits = NC * UPT;
     constexpr int kTileBytes = kTileUnits * kUnitBytes;
+    // 16-bit draws with the 2 x 512 tile: a thread's two units are 512 apart in a 1024-aligned tile,
+    // i.e. the two halves of one pair, so one Philox block per worker serves both.
+    constexpr bool kPairShared = ROUND == INTSGD_ROUND_RANDOM16 && NC == 512 && UPT == 2;
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(16) uint4 s_tab[INTSGD_MAX_WORKERS];
     __shared__ uint64_t full_bar[NS], empty_bar[NS];
@@ -236,6 +243,15 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         const float alpha = st->alpha, cdec = st->c;
         const uint32_t step = st->step;
         const BlockParams& bp = P.bp;
+        auto unit_draws = [&](const PhiloxThreadPart& t, const uint4& e, const uint4& pw, int k, bool h) -> uint4 {
+            if (ROUND == INTSGD_ROUND_RANDOM) return philox_finish(t, e, P.keys);
+            if (ROUND == INTSGD_ROUND_RANDOM16) {
+                if (kPairShared) return k == 0 ? split16(pw.x, pw.y) : split16(pw.z, pw.w);
+                const uint4 r = philox_finish(t, e, P.keys);
+                return h ? split16(r.z, r.w) : split16(r.x, r.y);
+            }
+            return make_uint4(0, 0, 0, 0);
+        };
         uint32_t s = 0, phase = 0;
         float max_sum = 0.0f;                                            // max |S| over fast-path units
         const bool count_overflow = P.agg_limit != 0x7FFFFFFF;          // int8 wire: count |S| > 127
@@ -246,15 +262,18 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
             UnitAcc ua[UPT];
             float2 a01[UPT], a23[UPT];
             int s_lo[UPT], s_hi[UPT];
-            bool active[UPT];
+            bool active[UPT], half[UPT];
 #pragma unroll
             for (int k = 0; k < UPT; ++k) {
                 const int64_t unit = unit0 + (int64_t)k * NC;
                 active[k] = unit < PP.units;
+                half[k] = (unit >> 9) & 1;
                 xo[k] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (active[k]) xo[k] = load_f4<true>(P.x, unit);
                 tp[k].n3 = tp[k].H = tp[k].m1 = 0;
                 if (ROUND == INTSGD_ROUND_RANDOM) tp[k] = philox_thread_part((uint32_t)unit, step, P.keys);
+                if (ROUND == INTSGD_ROUND_RANDOM16 && !(kPairShared && k > 0))
+                    tp[k] = philox_thread_part(pair_index((uint32_t)unit), step, P.keys);
                 ua[k].F01 = make_float2(0.f, 0.f);
                 ua[k].F23 = make_float2(0.f, 0.f);
                 ua[k].m = 0.0f;
@@ -282,24 +301,24 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
 #pragma unroll
                     for (int w = 0; w < G; ++w) {
                         const uint4 e = s_tab[g0 + w];
+                        uint4 pw = make_uint4(0, 0, 0, 0);
+                        if (kPairShared) pw = philox_finish(tp[0], e, P.keys);   // one block for both units
 #pragma unroll
                         for (int k = 0; k < UPT; ++k) {
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
-                            uint4 rw = make_uint4(0, 0, 0, 0);
-                            if (ROUND == INTSGD_ROUND_RANDOM) rw = philox_finish(tp[k], e, P.keys);
-                            consume_unit<ROUND>(gv, a01[k], a23[k], rw, ua[k]);
+                            consume_unit<ROUND>(gv, a01[k], a23[k], unit_draws(tp[k], e, pw, k, half[k]), ua[k]);
                         }
                     }
                 } else {
                     for (int w = 0; w < gw; ++w) {
                         const uint4 e = s_tab[g0 + w];
+                        uint4 pw = make_uint4(0, 0, 0, 0);
+                        if (kPairShared) pw = philox_finish(tp[0], e, P.keys);
 #pragma unroll
                         for (int k = 0; k < UPT; ++k) {
                             if (!active[k]) continue;
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
-                            uint4 rw = make_uint4(0, 0, 0, 0);
-                            if (ROUND == INTSGD_ROUND_RANDOM) rw = philox_finish(tp[k], e, P.keys);
-                            consume_unit<ROUND>(gv, a01[k], a23[k], rw, ua[k]);
+                            consume_unit<ROUND>(gv, a01[k], a23[k], unit_draws(tp[k], e, pw, k, half[k]), ua[k]);
                         }
                     }
                 }
@@ -388,8 +407,8 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 int S = 0;
                 for (int i = 0; i < n; ++i) {
                     uint32_t word = 0;
-                    if (ROUND == INTSGD_ROUND_RANDOM) {
-                        const uint4 w4 = draw_unit(j >> 2, (uint32_t)i, step, P.keys);
+                    if (ROUND != INTSGD_ROUND_NEAREST) {
+                        const uint4 w4 = draw_unit<ROUND>(j >> 2, (uint32_t)i, step, P.keys);
                         const uint32_t wv[4] = {w4.x, w4.y, w4.z, w4.w};
                         word = wv[j & 3];
                     }
