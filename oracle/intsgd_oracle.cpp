@@ -16,7 +16,7 @@
 // paper's order; there is no blocking, vectorisation or fusion.
 //
 // Pins (tests marked "not gpu"): Philox known-answer vectors; E[Int(t)] = t, |Int(t)-t| < 1,
-// Var <= 1/4 (Lemma 1); the decode identity below Eq. 2; the hand-worked 4-element alpha and
+// Var <= 1/4 (Lemma 1); floor(t + u) against exact rationals; the decode identity below Eq. 2; the hand-worked 4-element alpha and
 // encode/aggregate/update examples; the closed form d*eta^2/alpha^2 = eta^2 eps^2 + 2 n r
 // (proof of Proposition 2); Proposition 3 as the beta = eps = 0 special case; Algorithm 2 with
 // one block equal to Algorithm 1; brute force against exact rational arithmetic on tiny
@@ -91,9 +91,14 @@ float draw_uniform16(uint64_t seed, uint32_t step, uint32_t worker, uint64_t j) 
     return (float)v * 1.52587890625e-5f;  // 2^-16
 }
 
-// 24-bit uniform in [0, 1): the top 24 bits of the word times 2^-24; exact in fp32.
+// Uniform in [0, 1) from a 32-bit word: w * 2^-32 truncated (toward zero) to fp32, i.e. the word
+// with everything below its 24 leading significant bits cleared.  Always below 1 (at most
+// 1 - 2^-24), and exact in fp32 by construction.
 float uniform_from_word(uint32_t w) {
-    return (float)(w >> 8) * 5.9604644775390625e-8f;  // 2^-24
+    int len = 0;
+    while (len < 32 && (w >> len) != 0) ++len;           // number of significant bits of w
+    if (len > 24) w &= ~((1u << (len - 24)) - 1u);       // keep the 24 leading ones
+    return (float)w * 2.3283064365386963e-10f;           // 2^-32; at most 24 significant bits: exact
 }
 
 float widen_bf16(uint16_t h) {
@@ -116,12 +121,17 @@ float limit_as_float(int64_t L) {
 }
 
 // Int(t) of Section 2: floor(t) + 1 with probability t - floor(t), else floor(t); the floor
-// is toward minus infinity.  The draw is "up iff u < p" with p = fl32(t - floor(t)).
+// is toward minus infinity.  Realised as floor(t + u) with u uniform on [0, 1): the sum reaches
+// floor(t) + 1 exactly when u >= 1 - (t - floor(t)), an event of probability t - floor(t).
+// The sum is never rounded: with k = floor(t), "t + u >= k + 1" is decided as u >= (k + 1) - t in
+// fp64.  That difference lies in (0, 1] and is exact whenever |t| >= 2^-28 (its bits span at most
+// 2^0 .. 2^-51) and for every negative t above -1 (it is -t); for 0 <= t < 2^-28 it is within
+// 2^-28 of 1, above every possible u (u <= 1 - 2^-24), exactly as the unrounded difference is.
 // Returned as an integer-valued float (no clipping here).
 float int_round_random(float y, float u) {
-    const float f = std::floor(y);
-    const float p = y - f;
-    return f + ((u < p) ? 1.0f : 0.0f);
+    const float k = std::floor(y);
+    const double need = ((double)k + 1.0) - (double)y;
+    return ((double)u >= need) ? (float)((double)k + 1.0) : k;
 }
 
 // Deterministic variant named in Section 5.1 ("IntSGD (Determ.)"): round to nearest, ties
@@ -214,7 +224,7 @@ void orc_scale_block(int64_t d, int64_t d_l, int32_t n, double eta, double beta,
 // ---- Algorithm 1, "scale and round the local gradient": Int(alpha_k g_i) ----------------
 // One worker, coordinates [j0, j0 + count) of a vector whose element 0 is grad[0]
 // (grad, payload and u_inject are indexed relative to j0; the random stream by j0 + t).
-// grad_dtype 0 = fp32, 1 = bf16; payload_dtype 0 = int32, 1 = int8; rounding 0 = random (24-bit draws),
+// grad_dtype 0 = fp32, 1 = bf16; payload_dtype 0 = int32, 1 = int8; rounding 0 = random (one Philox word per draw),
 // 2 = random with the 16-bit draws of draw_uniform16,
 // 1 = nearest-even.  u_inject (nullable) replaces the Philox draw, for hand examples.
 void orc_encode(const void* grad, int grad_dtype, int64_t j0, int64_t count, float alpha,

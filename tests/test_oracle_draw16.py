@@ -59,7 +59,7 @@ def test_uniformity_and_independence():
 
 @pytest.mark.parametrize("t", [0.25, -0.25, 3.7, -2.9, 0.5, 1.0 / 3.0])
 def test_rounding_is_unbiased_to_the_draw_resolution(t):
-    """P(up) = ceil(p 2^16) / 2^16, so |E Int(t) - t| <= 2^-16 (zero when p is a multiple of 2^-16)."""
+    """P(up) = floor(p 2^16) / 2^16, so |E Int(t) - t| <= 2^-16 (zero when p is a multiple of 2^-16)."""
     N = 1 << 17
     grad = np.full(N, t, dtype=np.float32)
     q, clip, nonf = oracle.encode(grad, np.float32(1.0), worker=1, step=4, seed=99, n=4, rounding=ROUND_RANDOM16)
@@ -67,9 +67,9 @@ def test_rounding_is_unbiased_to_the_draw_resolution(t):
     p = t32 - math.floor(t32)
     assert set(np.unique(q)) <= {math.floor(t32), math.floor(t32) + 1}
     assert abs(q.mean() - t32) <= 4 * math.sqrt(p * (1 - p) / N) + 2.0**-16
-    # the decision is "up iff u < p" with u = v 2^-16, element by element
+    # the decision is floor(t + u) with u = v 2^-16, element by element (exact in fp64: 24 + 16 bits)
     u = np.array([oracle.draw_uniform16(99, 4, 1, j) for j in range(256)])
-    assert np.array_equal(q[:256], math.floor(t32) + (u < np.float32(p)).astype(int))
+    assert np.array_equal(q[:256], np.floor(np.float64(t32) + u).astype(int))
 
 
 def test_step_with_16_bit_draws_differs_from_the_default_stream_only_in_the_draws():

@@ -27,10 +27,13 @@ MUTANTS = [
     ("philox key schedule dropped", "        k0 += kWeyl0;\n", ""),
     ("counter: worker and step swapped", "(uint32_t)(b >> 32), worker, step}", "(uint32_t)(b >> 32), step, worker}"),
     ("counter: one block per coordinate", "const uint64_t b = j >> 2;", "const uint64_t b = j;"),
-    ("uniform uses 23 bits", "return (float)(w >> 8) * 5.9604644775390625e-8f;", "return (float)(w >> 9) * 5.9604644775390625e-8f;"),
-    ("draw: up iff u <= p", "return f + ((u < p) ? 1.0f : 0.0f);", "return f + ((u <= p) ? 1.0f : 0.0f);"),
-    ("draw: direction reversed", "return f + ((u < p) ? 1.0f : 0.0f);", "return f + ((u >= p) ? 1.0f : 0.0f);"),
-    ("floor replaced by truncation", "const float f = std::floor(y);", "const float f = std::trunc(y);"),
+    ("uniform keeps 23 bits", "if (len > 24) w &= ~((1u << (len - 24)) - 1u);", "if (len > 23) w &= ~((1u << (len - 23)) - 1u);"),
+    ("uniform rounded to nearest, not truncated", "    if (len > 24) w &= ~((1u << (len - 24)) - 1u);", "    "),
+    ("draw: a sum on an integer stays down", "return ((double)u >= need) ?", "return ((double)u > need) ?"),
+    ("draw: direction reversed", "return ((double)u >= need) ?", "return ((double)u < need) ?"),
+    ("draw: complement dropped", "const double need = ((double)k + 1.0) - (double)y;", "const double need = (double)y - (double)k;"),
+    ("draw: sum rounded to fp32 before the floor", "return ((double)u >= need) ? (float)((double)k + 1.0) : k;", "return std::floor(y + u);"),
+    ("floor replaced by truncation", "const float k = std::floor(y);", "const float k = std::trunc(y);"),
     ("nearest: ties away from zero", "return std::nearbyintf(y);", "return std::roundf(y);"),
     ("clip: NaN not zeroed", "    if (y != y) qf = 0.0f;\n", ""),
     ("clip: limit off by one", "if (y > Lf) qf = Lf;", "if (y > Lf) qf = Lf + 1.0f;"),
@@ -72,9 +75,10 @@ def _battery():
     """A compact selection of the pins; raises AssertionError on the first one that fails."""
     tp.test_known_answer_vectors(GOLDEN)
     tp.test_stream_layout()
-    tp.test_uniform_from_word_is_top_24_bits()
+    tp.test_uniform_from_word_is_the_word_truncated_to_fp32()
     tr.test_int_definition_against_exact_rationals()
     tr.test_negative_half_integers()
+    tr.test_floor_of_the_unrounded_sum_on_adversarial_values()
     tr.test_unbiased_and_variance_monte_carlo(0.25)
     tr.test_nearest_even()
     tr.test_clip_counts_closed_form_int8()

@@ -1,4 +1,6 @@
 """Pins for the oracle's random stream: Philox4x32-10 and the (seed, step, worker, index) layout."""
+from fractions import Fraction
+
 import numpy as np
 
 import oracle
@@ -64,12 +66,20 @@ def test_stream_layout():
         assert oracle.draw_word(seed, step, worker, j) == words[j % 4]
 
 
-def test_uniform_from_word_is_top_24_bits():
-    for w in [0, 1, 255, 256, 0xFFFFFFFF, 0x80000000, 0x12345678]:
+def test_uniform_from_word_is_the_word_truncated_to_fp32():
+    """u = w * 2^-32 rounded toward zero to fp32: u <= w / 2^32 < next fp32 above u, and u < 1."""
+    rng = np.random.default_rng(4)
+    words = [0, 1, 255, 256, 0xFFFFFF, 0x1000000, 0x1000001, 0x1FFFFFF, 0xFFFFFFFF, 0xFFFFFF00, 0xFFFFFF7F,
+             0x80000000, 0x800000FF, 0x12345678] + [int(w) for w in rng.integers(0, 2**32, 2000)]
+    for w in words:
         u = oracle.uniform_from_word(w)
-        assert u == (w >> 8) / 2.0**24
-        assert 0.0 <= u < 1.0
+        assert np.float32(u) == u and 0.0 <= u < 1.0
+        exact = Fraction(w, 2**32)
+        above = float(np.nextafter(np.float32(u), np.float32(2.0)))
+        assert Fraction(u) <= exact < Fraction(above), hex(w)
     assert oracle.uniform_from_word(0xFFFFFFFF) == 1.0 - 2.0**-24
+    assert oracle.uniform_from_word(0xFFFFFF) == 0xFFFFFF / 2.0**32      # 24 significant bits: kept whole
+    assert oracle.uniform_from_word(0x1FFFFFF) == 0x1FFFFFE / 2.0**32    # 25 bits: the lowest one dropped
 
 
 def _draws(seed, step, worker, count, j0=0):

@@ -16,23 +16,55 @@ def test_int_of_integers_is_identity():
 
 
 def test_int_definition_against_exact_rationals():
-    # brute force: dyadic t (exact in fp32) x a grid of u; floor and the comparison in Fractions
+    # brute force: dyadic t (exact in fp32) x a grid of u; Int(t) = floor(t + u) in Fractions
     for num in range(-40, 41):
         t = Fraction(num, 8)
-        fl = math.floor(t)
-        p = t - fl
         for k in range(0, 16):
             u = Fraction(k, 16)
-            want = fl + (1 if u < p else 0)
+            want = math.floor(t + u)
             assert oracle.int_round(float(t), float(u)) == want, (t, u)
+            # the same event stated on the fractional part: up iff u >= 1 - (t - floor(t))
+            assert want == math.floor(t) + (1 if u >= 1 - (t - math.floor(t)) else 0)
+
+
+def test_floor_of_the_unrounded_sum_on_adversarial_values():
+    """t + u is never rounded before the floor: random and near-integer fp32 values with draws on
+    the 2^-32 grid, against exact rational arithmetic."""
+    rng = np.random.default_rng(8)
+    ts = [np.float32(v) for v in rng.normal(0, 100, 3000)] + [np.float32(v) for v in rng.normal(0, 1e-3, 500)]
+    for base in [1.0, -1.0, 100.0, -100.0, 4096.0, 2.0**20, -(2.0**22), 0.0]:
+        b = np.float32(base)
+        for _ in range(6):
+            ts += [b]
+            b = np.nextafter(b, np.float32(-np.inf), dtype=np.float32)
+        b = np.float32(base)
+        for _ in range(6):
+            b = np.nextafter(b, np.float32(np.inf), dtype=np.float32)
+            ts += [b]
+    ts += [np.float32(v) for v in [1e-10, -1e-10, 1e-38, -1e-38, 1e-45, -1e-45, 2.0**-28, -(2.0**-28), 2.0**-29, 2.0**-24, -(2.0**-24)]]
+    words = [0, 1, 2, 255, 256, 2**15 - 1, 2**24 - 1, 2**24, 2**31, 2**32 - 256, 2**32 - 1] + \
+            [int(w) for w in rng.integers(0, 2**32, 24)]
+    us = [oracle.uniform_from_word(w) for w in words]
+    for t in ts:
+        ft = Fraction(float(t))
+        for u in us:
+            assert oracle.int_round(float(t), u) == math.floor(ft + Fraction(u)), (float(t), u)
+        # the complement of the fractional part, and its fp32 neighbours, as draws (when they are valid draws)
+        need = 1 - (ft - math.floor(ft))
+        for cand in [np.float32(float(need))]:
+            for u in [np.nextafter(cand, np.float32(0)), cand, np.nextafter(cand, np.float32(2))]:
+                if 0 <= float(u) < 1:
+                    assert oracle.int_round(float(t), float(u)) == math.floor(ft + Fraction(float(u))), (float(t), float(u))
 
 
 def test_negative_half_integers():
     # Int(-1.5) is -2 or -1, each with probability 1/2: floor is toward minus infinity
-    assert oracle.int_round(-1.5, 0.49) == -1
-    assert oracle.int_round(-1.5, 0.5) == -2
-    assert oracle.int_round(-0.25, 0.74) == 0
-    assert oracle.int_round(-0.25, 0.75) == -1
+    assert oracle.int_round(-1.5, 0.49) == -2
+    assert oracle.int_round(-1.5, 0.5) == -1
+    assert oracle.int_round(-0.25, 0.24) == -1
+    assert oracle.int_round(-0.25, 0.25) == 0
+    assert oracle.int_round(0.75, 0.24) == 0
+    assert oracle.int_round(0.75, 0.25) == 1
 
 
 def test_error_strictly_below_one_everywhere():
@@ -57,6 +89,8 @@ def test_unbiased_and_variance_monte_carlo(t):
     p = t32 - math.floor(t32)
     sd = math.sqrt(p * (1 - p) / N)
     assert abs(q.mean() - t32) <= 4 * sd + 2.0**-24
+    if p not in (0.0,):
+        assert q.min() != q.max()      # both outcomes occur
     assert set(np.unique(q)) <= {math.floor(t32), math.floor(t32) + 1}
     assert q.var() <= 0.25 + 1e-12
     assert abs(q.var() - p * (1 - p)) < 0.01
@@ -86,10 +120,14 @@ def test_huge_values_round_to_themselves():
             assert oracle.int_round(y, u) == int(y)
 
 
-def test_tiny_negative_rounds_p_to_one():
-    # y = -1e-10: floor = -1 and fl32(y + 1) = 1, so the draw always goes up to 0
-    for u in [0.0, 0.5, 1.0 - 2.0**-24]:
+def test_tiny_values_are_not_rounded_away():
+    # y = -1e-10: floor = -1; any positive draw lifts the sum above 0, the zero draw does not
+    assert oracle.int_round(-1e-10, 0.0) == -1
+    for u in [2.0**-32, 0.5, 1.0 - 2.0**-24]:
         assert oracle.int_round(-1e-10, u) == 0
+    # y = +1e-10 never reaches 1: the largest draw is 1 - 2^-24
+    for u in [0.0, 0.5, 1.0 - 2.0**-24]:
+        assert oracle.int_round(1e-10, u) == 0
 
 
 def test_nearest_even():

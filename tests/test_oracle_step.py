@@ -54,9 +54,7 @@ def test_brute_force_tiny_against_exact_rationals():
             for u in product(grid_u, repeat=n):
                 S = 0
                 for gi, ui in zip(g, u):
-                    y = alpha * gi
-                    fl = math.floor(y)
-                    S += fl + (1 if ui < y - fl else 0)
+                    S += math.floor(alpha * gi + ui)      # Int(t) = floor(t + u)
                 x0 = Fraction(3, 4)
                 x_want = x0 - c * S
                 payloads = []
