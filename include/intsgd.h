@@ -25,9 +25,11 @@
  *    must be issued on one stream (or be ordered by the caller).
  *  - The random stream is counter-based: Philox4x32-10 (Salmon et al., SC'11) with
  *    key = (seed low, seed high), counter = (b low, b high, worker, step), b = j / 4, and
- *    coordinate j uses output word j mod 4.  u = (word >> 8) * 2^-24; Int rounds up iff
- *    u < fl32(y - floor(y)) with y = fl32(alpha * g).  Results do not depend on the launch shape.
- *  - fp32 arithmetic of the vector part is unfused (separately rounded multiply and subtract).
+ *    coordinate j uses output word j mod 4.  u = word * 2^-32 truncated to fp32 (its 24 leading
+ *    significant bits; u <= 1 - 2^-24); Int(y) = floor(y + u) evaluated on the unrounded sum, with
+ *    y = fl32(alpha * g): up with probability y - floor(y).  Results do not depend on the launch shape.
+ *  - fp32 arithmetic of the scale, decode and update steps is unfused (separately rounded multiply
+ *    and subtract).
  */
 #ifndef INTSGD_H_
 #define INTSGD_H_
@@ -64,7 +66,7 @@ extern "C" {
                                     P = ((u >> 10) << 9) | (u & 511) (counter (P low, P high, worker, step))
                                     with unit u ^ 512, takes words 2h and 2h + 1 (h = bit 9 of u); coordinate
                                     e = j mod 4 uses the low (e even) or high (e odd) 16 bits v of word
-                                    2h + e / 2; rounds up iff v * 2^-16 < fl32(y - floor(y)).  Bias at most
+                                    2h + e / 2; Int(y) = floor(y + v * 2^-16).  Bias at most
                                     2^-16 per value.  Halves the random-number work: an option, not the default */
 #define INTSGD_MODE_EXACT      0 /* Algorithm 1, Init line: x <- x - eta (1/n) sum_i g_i, uncompressed */
 #define INTSGD_MODE_TWO_KERNEL 1 /* encode every worker to a payload buffer, then aggregate */

@@ -293,7 +293,7 @@ int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     PP.units = units;
     PP.tiles = 0;   // set by the launcher from the tile shape
     if (ctx->bs.B > 0) fill_block_params(ctx, PP.v, units << 2);
-    // Floors and up-decisions are summed as integer-valued floats: exact while n * (T + 1) <= 2^24.
+    // Rounded values are summed as integer-valued floats: exact while n * (T + 1) <= 2^24.
     const float t_max = (float)((1 << 24) / ctx->cfg.n - 2);
     PP.fast_limit = ctx->Lf < t_max ? ctx->Lf : t_max;
     const int rounding = ctx->cfg.rounding;

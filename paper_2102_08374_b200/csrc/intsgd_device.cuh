@@ -102,8 +102,7 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 }
 
 // Random draws of unit `unit` (coordinates 4*unit .. 4*unit+3) of `worker` at `step`, one per
-// coordinate.  Default stream: the four words of Philox block `unit`; the rounding uses their top 24
-// bits.  INTSGD_ROUND_RANDOM16: 16-bit draws; unit u shares the block of pair index
+// coordinate.  Default stream: the four words of Philox block `unit`.  INTSGD_ROUND_RANDOM16: 16-bit draws; unit u shares the block of pair index
 // P = ((u >> 10) << 9) | (u & 511) with the unit 512 places away, takes words 2h and 2h + 1
 // (h = bit 9 of u), and coordinate e gets the low (e even) or high (e odd) half of word 2h + e / 2.
 template <int ROUND>
@@ -119,14 +118,15 @@ __device__ __forceinline__ uint4 draw_unit(int64_t unit, uint32_t worker, uint32
     return philox4x32_10((uint32_t)unit, (uint32_t)((uint64_t)unit >> 32), worker, step, K);
 }
 
-// The draw as a float and the power of two that scales the fractional part to the same range.
+// The uniform draw is draw_as_float(w) * draw_scale(): the word times 2^-32 truncated to fp32 (the
+// conversion rounds toward zero, so u <= 1 - 2^-24), or the 16-bit value times 2^-16.
 template <int ROUND>
 __device__ __forceinline__ float draw_as_float(uint32_t w) {
-    return (ROUND == INTSGD_ROUND_RANDOM16) ? __uint2float_rn(w) : __uint2float_rn(w >> 8);
+    return (ROUND == INTSGD_ROUND_RANDOM16) ? __uint2float_rn(w) : __uint2float_rz(w);
 }
 template <int ROUND>
 __device__ __forceinline__ float draw_scale() {
-    return (ROUND == INTSGD_ROUND_RANDOM16) ? 65536.0f : 16777216.0f;
+    return (ROUND == INTSGD_ROUND_RANDOM16) ? 1.52587890625e-05f : 2.3283064365386963e-10f;
 }
 
 // ----------------------------------------------------------------------------------------
@@ -191,27 +191,17 @@ __device__ __forceinline__ float absmax3_nan(float a, float b, float c) {
     return d;
 }
 
-// 1.0f if a < b else 0.0f, in one instruction.
-__device__ __forceinline__ float lt_as_float(float a, float b) {
-    float d;
-    asm("set.lt.f32.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
-    return d;
-}
-
 // ----------------------------------------------------------------------------------------
-// Rounding.  y = fl32(alpha * g).  Random: f = floor(y), p = fl32(y - f),
-// u = (w >> 8) * 2^-24, q = f + [u < p]  (Int(t), Section 2 of the paper).
-// The comparison is done as (float)(w >> 8) < p * 2^24: both scalings are exact.
-// (With 16-bit draws: (float)v < p * 2^16.)
+// Rounding.  y = fl32(alpha * g).  Random: q = floor(y + u) on the unrounded sum (Int(t), Section 2
+// of the paper: up with probability t - floor(t)).  One fused multiply-add rounded toward minus
+// infinity forms RD(y + u): the product draw * scale is exact, and rounding the sum down never crosses
+// an integer (every integer of the range is an fp32 value, or y is itself an integer and u < 1), so
+// floor(RD(y + u)) = floor(y + u).
 // ----------------------------------------------------------------------------------------
 template <int ROUND>
 __device__ __forceinline__ int round_in_range(float y, uint32_t w) {
     if (ROUND == INTSGD_ROUND_NEAREST) return __float2int_rn(y);
-    const float f = floorf(y);
-    const float p = __fsub_rn(y, f);
-    const float uf = draw_as_float<ROUND>(w);
-    const float pscaled = __fmul_rn(p, draw_scale<ROUND>());
-    return __float2int_rz(f) + (uf < pscaled ? 1 : 0);
+    return __float2int_rd(__fmaf_rd(draw_as_float<ROUND>(w), draw_scale<ROUND>(), y));
 }
 
 // Full rule with clipping: values outside [-Lf, Lf] saturate, NaN becomes 0, and the event is
@@ -250,21 +240,15 @@ __device__ __noinline__ int4 round_unit_checked(float y0, float y1, float y2, fl
     return q;
 }
 
-// Four in-range values at once with packed fp32x2 arithmetic; bit-identical to round_in_range on
-// each (the same separately rounded steps: floor, y - f, scaling by 2^24, compare, add).
+// Four in-range values at once with packed fp32x2 arithmetic; bit-identical to round_in_range on each.
 template <int ROUND>
 __device__ __forceinline__ int4 round4_in_range(float2 y01, float2 y23, uint4 w) {
     if (ROUND == INTSGD_ROUND_NEAREST)
         return make_int4(__float2int_rn(y01.x), __float2int_rn(y01.y), __float2int_rn(y23.x), __float2int_rn(y23.y));
-    const float2 f01 = make_float2(floorf(y01.x), floorf(y01.y));
-    const float2 f23 = make_float2(floorf(y23.x), floorf(y23.y));
-    const float2 neg1 = make_float2(-1.0f, -1.0f), scale = make_float2(draw_scale<ROUND>(), draw_scale<ROUND>());
-    const float2 p01 = __fmul2_rn(__ffma2_rn(f01, neg1, y01), scale);
-    const float2 p23 = __fmul2_rn(__ffma2_rn(f23, neg1, y23), scale);
-    const float2 u01 = make_float2(lt_as_float(draw_as_float<ROUND>(w.x), p01.x), lt_as_float(draw_as_float<ROUND>(w.y), p01.y));
-    const float2 u23 = make_float2(lt_as_float(draw_as_float<ROUND>(w.z), p23.x), lt_as_float(draw_as_float<ROUND>(w.w), p23.y));
-    const float2 q01 = __fadd2_rn(f01, u01), q23 = __fadd2_rn(f23, u23);
-    return make_int4(__float2int_rz(q01.x), __float2int_rz(q01.y), __float2int_rz(q23.x), __float2int_rz(q23.y));
+    const float2 scale = make_float2(draw_scale<ROUND>(), draw_scale<ROUND>());
+    const float2 z01 = __ffma2_rd(make_float2(draw_as_float<ROUND>(w.x), draw_as_float<ROUND>(w.y)), scale, y01);
+    const float2 z23 = __ffma2_rd(make_float2(draw_as_float<ROUND>(w.z), draw_as_float<ROUND>(w.w)), scale, y23);
+    return make_int4(__float2int_rd(z01.x), __float2int_rd(z01.y), __float2int_rd(z23.x), __float2int_rd(z23.y));
 }
 
 // One unit of one worker: scale, round, clip.  The common case (all four values in range) has no

@@ -58,7 +58,7 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
 }
 
 // ---- per-unit arithmetic ------------------------------------------------------------------------
-// Fast path of one worker's unit.  Floors and up-decisions are accumulated as integer-valued
+// Fast path of one worker's unit.  The rounded values are accumulated as integer-valued
 // floats (exact: the host caps the fast-path magnitude T so that n * (T + 1) <= 2^24, and T never
 // exceeds the clip limit); `m` tracks max |alpha g| (NaN-propagating) so that a unit with any value
 // outside the fast range -- clipped, huge or not finite -- is redone exactly at the end of its tile.
@@ -78,15 +78,12 @@ __device__ __forceinline__ void consume_unit(float4 g, float2 alpha01, float2 al
         u.F23 = __fadd2_rn(u.F23, make_float2(rintf(y23.x), rintf(y23.y)));
         return;
     }
-    const float2 f01 = make_float2(floorf(y01.x), floorf(y01.y));
-    const float2 f23 = make_float2(floorf(y23.x), floorf(y23.y));
-    const float2 neg1 = make_float2(-1.0f, -1.0f), scale = make_float2(draw_scale<ROUND>(), draw_scale<ROUND>());
-    const float2 p01 = __fmul2_rn(__ffma2_rn(f01, neg1, y01), scale);   // fl32(y - f) * 2^24 (2^16), both exact steps
-    const float2 p23 = __fmul2_rn(__ffma2_rn(f23, neg1, y23), scale);
-    const float2 u01 = make_float2(lt_as_float(draw_as_float<ROUND>(w.x), p01.x), lt_as_float(draw_as_float<ROUND>(w.y), p01.y));
-    const float2 u23 = make_float2(lt_as_float(draw_as_float<ROUND>(w.z), p23.x), lt_as_float(draw_as_float<ROUND>(w.w), p23.y));
-    u.F01 = __fadd2_rn(__fadd2_rn(u.F01, f01), u01);
-    u.F23 = __fadd2_rn(__fadd2_rn(u.F23, f23), u23);
+    // floor(y + u) on the unrounded sum: fused multiply-add rounded down, then floor (see round_in_range)
+    const float2 scale = make_float2(draw_scale<ROUND>(), draw_scale<ROUND>());
+    const float2 z01 = __ffma2_rd(make_float2(draw_as_float<ROUND>(w.x), draw_as_float<ROUND>(w.y)), scale, y01);
+    const float2 z23 = __ffma2_rd(make_float2(draw_as_float<ROUND>(w.z), draw_as_float<ROUND>(w.w)), scale, y23);
+    u.F01 = __fadd2_rn(u.F01, make_float2(floorf(z01.x), floorf(z01.y)));
+    u.F23 = __fadd2_rn(u.F23, make_float2(floorf(z23.x), floorf(z23.y)));
 }
 
 // Exact redo of one unit from global memory with the full clipping rule and the counters (rare:

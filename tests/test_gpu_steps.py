@@ -103,6 +103,36 @@ def test_values_outside_the_fast_range_clip_and_count_exactly(which, grad_dtype,
         ls.close()
 
 
+@pytest.mark.parametrize("which", [FUSED_PIPELINED, FUSED_DIRECT, TWO_KERNEL])
+@pytest.mark.parametrize("rounding", [pkg.ROUND_RANDOM, pkg.ROUND_RANDOM16])
+def test_values_next_to_integers_and_tiny_values(which, rounding):
+    """Int(y) = floor(y + u) must be taken on the unrounded sum: scaled gradients a few ulps from an
+    integer (both sides), exact integers, halves, and values down to the subnormals."""
+    n, d, eta, seed = 4, 2 * 4096 + 5, 0.1, 5
+    rng = np.random.default_rng(17)
+    mode, path = _mode_and_path(which)
+    ls = LockStep(n, d, rounding=rounding, seed=seed, x0=rng.normal(0, 1, d).astype(np.float32), fused_path=path)
+    try:
+        ls.exact([rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)], eta)
+        for k in range(3):
+            _, _, alpha, _ = oracle.scale(d, n, eta, ls.orc.beta, ls.orc.eps, ls.orc.r, ls.orc.dx2)
+            grads = []
+            for i in range(n):
+                ints = rng.integers(-200, 201, d).astype(np.float64)
+                off = rng.choice([0.0, 0.5, 2.0**-20, -(2.0**-20), 2.0**-16, -(2.0**-16), 2.0**-12, -(2.0**-12)], d)
+                g = ((ints + off) / float(alpha)).astype(np.float32)
+                for _ in range(2):      # and their fp32 neighbours
+                    idx = rng.integers(0, d, d // 8)
+                    g[idx] = np.nextafter(g[idx], np.float32(rng.choice([-1e9, 1e9])))
+                tiny = rng.integers(0, d, d // 16)
+                g[tiny] = (rng.choice([-1.0, 1.0], tiny.size) * 10.0 ** rng.uniform(-45, -6, tiny.size)).astype(np.float32)
+                grads.append(g)
+            st, ref = ls.step(grads, eta, mode=mode)
+            assert sum(st["clip_count"]) == 0
+    finally:
+        ls.close()
+
+
 @pytest.mark.parametrize("n,d", [(1, 1), (1, 5), (2, 3), (64, 1000), (3, 4), (16, 2), (2, 8), (3, 9), (5, 2049)])
 def test_degenerate_shapes(n, d):
     rng = np.random.default_rng(n * 1000 + d)
