@@ -38,6 +38,8 @@ struct intsgd_ctx {
     void* stage_grads[INTSGD_MAX_WORKERS];
     float* stage_x;
     int32_t* stage_agg;
+    cudaStream_t back_stream;   // device->host copies of finished windows (non-blocking stream)
+    cudaEvent_t window_done;
     char err[256];
 };
 
@@ -254,8 +256,9 @@ cudaError_t launch_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s)
         default: return launch_pipe_v<GRAD, ROUND, false, 0>(ctx, PP, s);
     }
 }
-bool pipe_eligible(const intsgd_ctx* ctx, bool aligned) {
-    const int64_t units = ctx->cfg.d >> 2;
+// `d` is the length of the launch (a window of the vector, or all of it).
+bool pipe_eligible(const intsgd_ctx* ctx, bool aligned, int64_t d) {
+    const int64_t units = d >> 2;
     return aligned && ctx->cfg.d <= ((int64_t)1 << 34) && units >= 2;
 }
 
@@ -288,7 +291,7 @@ int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     PP.v = P;
     PP.tab = ctx->tab;
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
-    int64_t units = ctx->cfg.d >> 2;
+    int64_t units = P.d >> 2;
     if (bf16) units &= ~(int64_t)1;   // bulk copies move multiples of 16 bytes
     PP.units = units;
     PP.tiles = 0;   // set by the launcher from the tile shape
@@ -324,9 +327,9 @@ void launch_fused_blocks_r(const intsgd_ctx* ctx, const VecParams& P, int grid, 
 }
 
 int launch_fused(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
-    const bool want_pipe = ctx->fused_path != 1 && pipe_eligible(ctx, aligned);
+    const bool want_pipe = ctx->fused_path != 1 && pipe_eligible(ctx, aligned, P.d);
     if (want_pipe) return launch_fused_pipe(ctx, P, s);
-    const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
+    const int grid = grid_for(ctx, (P.d + 3) / 4);
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
     if (ctx->bs.B > 0) {
         VecParams Q = P;
@@ -367,7 +370,7 @@ int launch_diana(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t
 }
 
 int launch_exact(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
-    const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
+    const int grid = grid_for(ctx, (P.d + 3) / 4);
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
     if (ctx->bs.B > 0) {
         VecParams Q = P;
@@ -403,6 +406,10 @@ void free_staging(intsgd_ctx* ctx) {
     }
     if (ctx->stage_x) cudaFree(ctx->stage_x);
     if (ctx->stage_agg) cudaFree(ctx->stage_agg);
+    if (ctx->back_stream) cudaStreamDestroy(ctx->back_stream);
+    if (ctx->window_done) cudaEventDestroy(ctx->window_done);
+    ctx->back_stream = nullptr;
+    ctx->window_done = nullptr;
     ctx->stage_x = nullptr;
     ctx->stage_agg = nullptr;
 }
@@ -751,6 +758,62 @@ int intsgd_heuristic_step(intsgd_ctx* ctx, const void* const* grads, float* x, i
     return rc;
 }
 
+// Host-buffer step over windows of the vector: window w is copied in, stepped and copied back while
+// window w + 1 is on its way in (the two directions of the link run at the same time).  The windows of
+// one step share the scale, the step index and the counters; the random stream is addressed by the
+// coordinate's index in the whole vector, so the integers and the iterate are those of a single launch,
+// and the squared step length is the sum of the windows' sums.
+constexpr int64_t kHostWindow = (int64_t)1 << 22;   // coordinates; a multiple of 4096 (whole tiles and draw pairs)
+
+static int step_host_windowed(intsgd_ctx* ctx, const void* const* host_grads, float* host_x, int32_t* host_agg,
+                              double eta_k, int32_t mode, cudaStream_t s) {
+    if (!(eta_k > 0.0) || !std::isfinite(eta_k)) return fail(ctx, INTSGD_ERR_INVALID_ARG, "eta_k must be finite and > 0");
+    if (mode != INTSGD_MODE_EXACT && mode != INTSGD_MODE_FUSED) return fail(ctx, INTSGD_ERR_INVALID_ARG, "bad mode");
+    if (!ctx->back_stream) {
+        CUDA_TRY(ctx, cudaStreamCreateWithFlags(&ctx->back_stream, cudaStreamNonBlocking));
+        CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->window_done, cudaEventDisableTiming));
+    }
+    const int n = ctx->cfg.n;
+    const int64_t d = ctx->cfg.d;
+    const size_t gsz = grad_elem_size(ctx->cfg.grad_dtype);
+    const bool want_agg = host_agg && mode != INTSGD_MODE_EXACT;
+    ctx->last_stream = s;
+    int rc;
+    if (mode == INTSGD_MODE_FUSED && (rc = launch_scale(ctx, eta_k, -1.0, s)) != INTSGD_OK) return rc;
+    for (int64_t off = 0; off < d; off += kHostWindow) {
+        const int64_t len = (d - off < kHostWindow) ? d - off : kHostWindow;
+        VecParams P;
+        base_params(ctx, P);
+        P.d = len;
+        P.unit_base = off >> 2;
+        P.window_flags = (off > 0 ? kWindowAccumulate : 0) | (off + len < d ? kWindowHoldStep : 0);
+        for (int i = 0; i < n; ++i) {
+            char* dst = (char*)ctx->stage_grads[i] + (size_t)off * gsz;
+            CUDA_TRY(ctx, cudaMemcpyAsync(dst, (const char*)host_grads[i] + (size_t)off * gsz, (size_t)len * gsz,
+                                          cudaMemcpyHostToDevice, s));
+            P.in[i] = dst;
+        }
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->stage_x + off, host_x + off, (size_t)len * sizeof(float), cudaMemcpyHostToDevice, s));
+        P.x = ctx->stage_x + off;
+        P.agg = want_agg ? ctx->stage_agg + off : nullptr;
+        if (mode == INTSGD_MODE_EXACT) {
+            P.c_exact = (float)(eta_k / (double)n);
+            rc = launch_exact(ctx, P, true, s);
+        } else {
+            rc = launch_fused(ctx, P, true, s);
+        }
+        if (rc != INTSGD_OK) return rc;
+        CUDA_TRY(ctx, cudaEventRecord(ctx->window_done, s));
+        CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->back_stream, ctx->window_done, 0));
+        CUDA_TRY(ctx, cudaMemcpyAsync(host_x + off, ctx->stage_x + off, (size_t)len * sizeof(float), cudaMemcpyDeviceToHost,
+                                      ctx->back_stream));
+        if (want_agg)
+            CUDA_TRY(ctx, cudaMemcpyAsync(host_agg + off, ctx->stage_agg + off, (size_t)len * sizeof(int32_t),
+                                          cudaMemcpyDeviceToHost, ctx->back_stream));
+    }
+    return INTSGD_OK;
+}
+
 int intsgd_step_host(intsgd_ctx* ctx, const void* const* host_grads, float* host_x, int32_t* host_agg,
                      double eta_k, int32_t mode, void* stream) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
@@ -768,6 +831,13 @@ int intsgd_step_host(intsgd_ctx* ctx, const void* const* host_grads, float* host
         CUDA_TRY(ctx, cudaMalloc(&ctx->stage_agg, d * sizeof(int32_t)));
     }
     cudaStream_t s = (cudaStream_t)stream;
+    if (d > (size_t)kHostWindow && ctx->bs.B == 0) {
+        const int rc = step_host_windowed(ctx, host_grads, host_x, host_agg, eta_k, mode, s);
+        if (rc != INTSGD_OK) return rc;
+        CUDA_TRY(ctx, cudaStreamSynchronize(ctx->back_stream));
+        CUDA_TRY(ctx, cudaStreamSynchronize(s));
+        return INTSGD_OK;
+    }
     for (int i = 0; i < n; ++i)
         CUDA_TRY(ctx, cudaMemcpyAsync(ctx->stage_grads[i], host_grads[i], gbytes, cudaMemcpyHostToDevice, s));
     CUDA_TRY(ctx, cudaMemcpyAsync(ctx->stage_x, host_x, d * sizeof(float), cudaMemcpyHostToDevice, s));

@@ -60,6 +60,9 @@ struct BlockParams {
     int32_t B;
 };
 
+constexpr int kWindowAccumulate = 1;   // state.dx2 += this launch's sum (not the first window of the step)
+constexpr int kWindowHoldStep = 2;     // do not advance the step counter (not the last window of the step)
+
 struct VecParams {
     const void* in[INTSGD_MAX_WORKERS];   // gradients (encode / fused / exact) or payloads (aggregate)
     void* out[INTSGD_MAX_WORKERS];        // payloads (encode)
@@ -76,6 +79,12 @@ struct VecParams {
     float Lf;                             // clip limit as the largest fp32 <= L
     float c_exact;                        // exact step: fp32(eta / n)
     int32_t agg_limit;                    // coordinates with |S| above this count as agg_overflow
+    // A launch may cover a window of the vector (pointers and d describe the window): unit_base is the
+    // index of its first unit in the whole vector (random stream), and the flags chain the windows of
+    // one step: every window but the first adds its norm partial to the state, every window but the
+    // last leaves the step counter alone.
+    int64_t unit_base;
+    int32_t window_flags;
     PhiloxKeys keys;
     BlockParams bp;
 };
@@ -324,7 +333,7 @@ __device__ __forceinline__ void flush_sum_counters(const ThreadAcc& a, DevState*
 }
 
 __device__ __forceinline__ void grid_finalize(const ThreadAcc& a, DevState* st, double* partials,
-                                              bool advance_step) {
+                                              bool advance_step, int window_flags = 0) {
     __shared__ double s_warp[32];
     __shared__ bool s_last;
     flush_sum_counters(a, st);
@@ -342,8 +351,8 @@ __device__ __forceinline__ void grid_finalize(const ThreadAcc& a, DevState* st, 
     for (unsigned b = threadIdx.x; b < gridDim.x; b += blockDim.x) v += __ldcg(&partials[b]);
     const double total = block_tree(v, s_warp);
     if (threadIdx.x == 0) {
-        st->dx2 = total;
-        if (advance_step) st->step += 1;
+        st->dx2 = (window_flags & kWindowAccumulate) ? st->dx2 + total : total;
+        if (advance_step && !(window_flags & kWindowHoldStep)) st->step += 1;
         st->ticket = 0;
     }
 }

@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(kMaxThreads) fused_step_kernel(const __grid_co
         for (int i = 0; i < n; ++i) {
             const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, (uint32_t)i, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit + P.unit_base, (uint32_t)i, step, P.keys);
             const int4 q = round_unit<ROUND>(gv, alpha, w, P.Lf, &s_cnt[i], nonf_slot);
             S.x += q.x; S.y += q.y; S.z += q.z; S.w += q.w;
         }
@@ -275,7 +275,7 @@ __global__ void __launch_bounds__(kMaxThreads) fused_step_kernel(const __grid_co
         int S[4] = {0, 0, 0, 0};
         for (int i = 0; i < n; ++i) {
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(full, (uint32_t)i, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(full + P.unit_base, (uint32_t)i, step, P.keys);
             const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
             for (int e = 0; e < tail; ++e) {
                 const float y = __fmul_rn(alpha, grad_at<GRAD>(P.in[i], 4 * full + e));
@@ -285,7 +285,7 @@ __global__ void __launch_bounds__(kMaxThreads) fused_step_kernel(const __grid_co
         for (int e = 0; e < tail; ++e) apply_coord(P, 4 * full + e, S[e], c, acc);
     }
     counters_flush(s_cnt, st);
-    grid_finalize(acc, st, P.partials, true);
+    grid_finalize(acc, st, P.partials, true, P.window_flags);
 }
 
 // ----------------------------------------------------------------------------------------
@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(kMaxThreads) exact_step_kernel(const __grid_co
             P.x[j] = exact_coord(P.x[j], m, c0, acc.dx2);
         }
     }
-    grid_finalize(acc, P.st, P.partials, true);
+    grid_finalize(acc, P.st, P.partials, true, P.window_flags);
 }
 
 // ----------------------------------------------------------------------------------------

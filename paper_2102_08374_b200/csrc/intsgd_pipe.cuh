@@ -95,7 +95,7 @@ __device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float4 
     for (int i = 0; i < P.n; ++i) {
         const float4 g = load_grad4<GRAD, true>(P.in[i], unit);
         uint4 w = make_uint4(0, 0, 0, 0);
-        if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, (uint32_t)i, step, P.keys);
+        if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit + P.unit_base, (uint32_t)i, step, P.keys);
         uint32_t clipped = 0, nonfinite = 0;
         S[0] += round_full<ROUND>(__fmul_rn(av[0], g.x), w.x, P.Lf, clipped, nonfinite);
         S[1] += round_full<ROUND>(__fmul_rn(av[1], g.y), w.y, P.Lf, clipped, nonfinite);
@@ -264,13 +264,13 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
             for (int k = 0; k < UPT; ++k) {
                 const int64_t unit = unit0 + (int64_t)k * NC;
                 active[k] = unit < PP.units;
-                half[k] = (unit >> 9) & 1;
+                half[k] = ((unit + P.unit_base) >> 9) & 1;
                 xo[k] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (active[k]) xo[k] = load_f4<true>(P.x, unit);
                 tp[k].n3 = tp[k].H = tp[k].m1 = 0;
-                if (ROUND == INTSGD_ROUND_RANDOM) tp[k] = philox_thread_part((uint32_t)unit, step, P.keys);
+                if (ROUND == INTSGD_ROUND_RANDOM) tp[k] = philox_thread_part((uint32_t)(unit + P.unit_base), step, P.keys);
                 if (ROUND == INTSGD_ROUND_RANDOM16 && !(kPairShared && k > 0))
-                    tp[k] = philox_thread_part(pair_index((uint32_t)unit), step, P.keys);
+                    tp[k] = philox_thread_part(pair_index((uint32_t)(unit + P.unit_base)), step, P.keys);
                 ua[k].F01 = make_float2(0.f, 0.f);
                 ua[k].F23 = make_float2(0.f, 0.f);
                 ua[k].m = 0.0f;
@@ -405,7 +405,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 for (int i = 0; i < n; ++i) {
                     uint32_t word = 0;
                     if (ROUND != INTSGD_ROUND_NEAREST) {
-                        const uint4 w4 = draw_unit<ROUND>(j >> 2, (uint32_t)i, step, P.keys);
+                        const uint4 w4 = draw_unit<ROUND>((j >> 2) + P.unit_base, (uint32_t)i, step, P.keys);
                         const uint32_t wv[4] = {w4.x, w4.y, w4.z, w4.w};
                         word = wv[j & 3];
                     }
@@ -427,7 +427,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
     counters_flush(s_cnt, st);   // includes a __syncthreads()
     if (threadIdx.x == 0 && s_fault) atomicExch(&st->fault, 1);
     if (BLOCKS) flush_sum_counters(acc, st);   // the per-segment norms are finished by block_norm_kernel
-    else grid_finalize(acc, st, P.partials, true);
+    else grid_finalize(acc, st, P.partials, true, P.window_flags);
 }
 
 }  // namespace intsgd

@@ -226,3 +226,40 @@ def test_step_host_matches_the_device_path():
         sb = b.intsgd_get_stats()
     assert np.array_equal(hx.numpy(), to_host(xa)) and np.array_equal(hagg.numpy(), to_host(agg_a))
     assert sa["dx2"] == sb["dx2"] and sa["alpha"] == sb["alpha"]
+
+
+@pytest.mark.parametrize("grad_dtype,rounding", [(pkg.GRAD_F32, pkg.ROUND_RANDOM), (pkg.GRAD_BF16, pkg.ROUND_RANDOM16)])
+def test_step_host_over_several_windows_matches_the_oracle(grad_dtype, rounding):
+    """A vector longer than the host path's window (2^22 coordinates) is stepped window by window with
+    the copies overlapped; integers and iterate must be those of the single-launch definition."""
+    n, d, seed, eta = 2, 2 * (1 << 22) + 4101, 13, 0.1
+    rng = np.random.default_rng(19)
+
+    def grads():
+        out = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
+        return [synth.to_bf16_bits(g) for g in out] if grad_dtype == pkg.GRAD_BF16 else out
+
+    x0 = rng.normal(0, 1, d).astype(np.float32)
+    orc = oracle.OracleIntSGD(n, d, seed=seed, rounding=rounding)
+    x_ref = x0.copy()
+    with pkg.IntSGD(n, d, grad_dtype=grad_dtype, seed=seed, rounding=rounding) as lib:
+        hx = torch.from_numpy(x0.copy()).pin_memory()
+        hagg = torch.zeros(d, dtype=torch.int32).pin_memory()
+        g = grads()
+        pin = lambda a: torch.from_numpy(a.view(np.int16).copy() if a.dtype == np.uint16 else a.copy()).pin_memory()
+        hg = [pin(a) for a in g]
+        lib.intsgd_step_host(hg, hx, None, eta_k=eta, mode=pkg.MODE_EXACT)
+        ref = orc.exact_step(g, x_ref, eta)
+        st = lib.intsgd_get_stats()
+        assert np.array_equal(hx.numpy(), x_ref) and rel_close(st["dx2"], ref["dx2"]) and st["step"] == 1
+        for k in range(2):
+            g = grads()
+            hg = [pin(a) for a in g]
+            lib.intsgd_step_host(hg, hx, hagg, eta_k=eta, mode=pkg.MODE_FUSED)
+            st = lib.intsgd_get_stats()
+            ref = orc.int_step(g, x_ref, eta, alpha_c=(np.float32(st["alpha"]), np.float32(st["c"])))
+            assert rel_close(st["alpha"], float(ref["alpha"])) and rel_close(st["r"], ref["r"])
+            assert np.array_equal(hagg.numpy(), ref["agg"])
+            assert np.array_equal(hx.numpy().view(np.uint32), x_ref.view(np.uint32))
+            assert rel_close(st["dx2"], ref["dx2"]) and st["max_abs_agg"] == ref["max_abs_agg"]
+            assert st["clip_count"] == ref["clip_count"] and st["step"] == k + 2
