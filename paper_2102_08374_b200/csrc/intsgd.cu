@@ -236,7 +236,8 @@ constexpr int kNumPipeShapes = sizeof(kPipeShapes) / sizeof(kPipeShapes[0]);
 
 template <int GRAD, int ROUND, bool BLOCKS, int V>
 cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
-    constexpr PipeShape S = kPipeShapes[V];
+    // bf16 tiles are half as large: the default shape stages 8 worker tiles at a time (fewer barrier rounds)
+    constexpr PipeShape S = (GRAD == INTSGD_GRAD_BF16 && V == 0) ? PipeShape{512, 2, 8, 3} : kPipeShapes[V];
     auto kernel = fused_pipe_kernel<GRAD, ROUND, BLOCKS, S.nc, S.upt, S.g, S.ns>;
     const int unit_bytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
     const int smem = S.ns * S.g * S.nc * S.upt * unit_bytes;
