@@ -33,8 +33,8 @@ HBM_FALLBACK_GBS = 6650.0
 # command and figures in profiles/fused_pipe_kernel_d24_n16_ncu_full.md): bytes per coordinate of the
 # captured case (d = 2^24, n = 16, fp32, int32 aggregate), valid for the kernel sources with this hash.
 # Any change to the kernel sources makes `roofline.traffic` null until the counters are taken again.
-NCU_TRAFFIC = {"sources_sha256": "bb6be72ac34aa26293852d713466a102b4a50ba2b933515ee1620b4cd32ea8cf",
-               "bytes_per_coordinate": 1.266304e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
+NCU_TRAFFIC = {"sources_sha256": "398ec93cee829894ff001ee38c4035fbbff4e7ab432ac913cba4763b3fa1121f",
+               "bytes_per_coordinate": 1.265483e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
 
 
 def kernel_sources_hash():
@@ -67,7 +67,8 @@ def parse_args():
     p.add_argument("--payload", default="int32", choices=["int32", "int8"])
     p.add_argument("--grad", default="f32", choices=["f32", "bf16"])
     p.add_argument("--mode", default="fused", choices=["fused", "two_kernel"])
-    p.add_argument("--rounding", default="random", choices=["random", "nearest"])
+    p.add_argument("--rounding", default="random", choices=["random", "nearest", "random16"],
+                   help="random16 = the optional 16-bit draw stream (a different random stream; not the default)")
     p.add_argument("--eta", type=float, default=0.1)
     p.add_argument("--e2e-steps", type=int, default=3)
     p.add_argument("--cpu-sample-log2", type=int, default=24,
@@ -162,7 +163,7 @@ def oracle_sample_throughput(n, d, sample_log2, grad_dtype, payload, rounding, s
         grads = [synth.to_bf16_bits(g) for g in grads]
     x = synth.iterate(w)
     pd = oracle.PAYLOAD_I8 if payload == "int8" else oracle.PAYLOAD_I32
-    rd = oracle.ROUND_NEAREST if rounding == "nearest" else oracle.ROUND_RANDOM
+    rd = {"nearest": oracle.ROUND_NEAREST, "random16": oracle.ROUND_RANDOM16}.get(rounding, oracle.ROUND_RANDOM)
     oracle.step_window([g[:1024] for g in grads], x[:1024].copy(), np.float32(700.0), np.float32(1e-5), step=1,
                        seed=seed, payload_dtype=pd, rounding=rd)     # load the library, touch the code
     t = time.perf_counter()
@@ -232,7 +233,7 @@ def main():
     n, d = args.workers, 1 << args.log2d
     grad_dtype = pkg.GRAD_BF16 if args.grad == "bf16" else pkg.GRAD_F32
     payload_dtype = pkg.PAYLOAD_I8 if args.payload == "int8" else pkg.PAYLOAD_I32
-    rounding = pkg.ROUND_NEAREST if args.rounding == "nearest" else pkg.ROUND_RANDOM
+    rounding = {"nearest": pkg.ROUND_NEAREST, "random16": pkg.ROUND_RANDOM16}.get(args.rounding, pkg.ROUND_RANDOM)
     mode = pkg.MODE_TWO_KERNEL if args.mode == "two_kernel" else pkg.MODE_FUSED
     gb, pb = (2 if args.grad == "bf16" else 4), (1 if args.payload == "int8" else 4)
 
