@@ -87,14 +87,14 @@ def _draws(seed, step, worker, count, j0=0):
 
 
 def test_uniformity_chi_square():
-    # 2^16 draws into 64 bins of the 24-bit uniform: chi-square with 63 dof, mean 63, sd ~11.2
+    # 2^16 draws into 64 bins by the word's top 6 bits: chi-square with 63 dof, mean 63, sd ~11.2
     w = _draws(seed=11, step=1, worker=0, count=1 << 16)
     bins = np.bincount((w >> 26).astype(np.int64), minlength=64)
     expect = (1 << 16) / 64
     chi2 = float(((bins - expect) ** 2 / expect).sum())
     assert 25.0 < chi2 < 120.0
-    # every bit of the 24 used ones is balanced (|mean - 1/2| < 5 sigma)
-    for bit in range(8, 32):
+    # every bit of the word is balanced (|mean - 1/2| < 5 sigma)
+    for bit in range(0, 32):
         frac = float(((w >> bit) & 1).mean())
         assert abs(frac - 0.5) < 5 * 0.5 / np.sqrt(len(w))
 
