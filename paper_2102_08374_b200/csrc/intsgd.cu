@@ -268,6 +268,7 @@ void fill_block_params(const intsgd_ctx* ctx, VecParams& P, int64_t covered_end)
     P.bp.alpha = ctx->bs.alpha;
     P.bp.c = ctx->bs.c;
     P.bp.chunk_sum = ctx->bs.chunk_sum;
+    P.bp.chunk_seg = ctx->bs.chunk_seg;
     P.bp.edge_sum = ctx->bs.edge_sum;
     P.bp.tail_sq = ctx->bs.tail_sq;
     P.bp.covered_end = covered_end;
@@ -926,10 +927,17 @@ int intsgd_set_blocks(intsgd_ctx* ctx, int32_t num_blocks, const int64_t* offset
     CUDA_TRY(ctx, cudaMalloc(&ctx->d_offsets, (B + 1) * sizeof(int64_t)));
     cudaError_t e = cudaMalloc(&base, bytes);
     double* chunk = nullptr;
-    if (e == cudaSuccess) e = cudaMalloc((void**)&chunk, chunks * sizeof(double));
+    // chunk partials (double) followed by the chunk -> segment table (int32)
+    if (e == cudaSuccess) e = cudaMalloc((void**)&chunk, chunks * (sizeof(double) + sizeof(int32_t)));
     if (e == cudaSuccess) e = cudaMemset(base, 0, bytes);
     if (e == cudaSuccess) e = cudaMemset(chunk, 0, chunks * sizeof(double));
     if (e == cudaSuccess) e = cudaMemcpy(ctx->d_offsets, offsets, (B + 1) * sizeof(int64_t), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) {
+        chunk_table_kernel<<<(unsigned)((chunks + 255) / 256), 256>>>(ctx->d_offsets, num_blocks, ctx->cfg.d,
+                                                                      reinterpret_cast<int32_t*>(chunk + chunks), (int64_t)chunks);
+        e = cudaGetLastError();
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    }
     // covered ranges: whole units of 4 (direct kernels, fp32 pipelined) and pairs of units (bf16 pipelined)
     const int64_t cov0 = (ctx->cfg.d >> 2) << 2, cov1 = (ctx->cfg.d >> 3) << 3;
     if (e == cudaSuccess) e = build_norm_plan(offsets, num_blocks, cov0, &ctx->plan[0], &ctx->d_plan_mem[0]);
@@ -956,6 +964,7 @@ int intsgd_set_blocks(intsgd_ctx* ctx, int32_t num_blocks, const int64_t* offset
     ctx->bs.alpha = reinterpret_cast<float*>(dbl + 4 * B + kMaxTail);
     ctx->bs.c = ctx->bs.alpha + B;
     ctx->bs.chunk_sum = chunk;
+    ctx->bs.chunk_seg = reinterpret_cast<int32_t*>(chunk + chunks);
     ctx->bs.B = num_blocks;
     return INTSGD_OK;
 }

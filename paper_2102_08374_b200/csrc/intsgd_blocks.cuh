@@ -37,13 +37,38 @@ struct UnitScale {
     int seg[4];
 };
 
-// Segment range [s_lo, s_hi] of the chunk that starts at unit `chunk_unit0` (warp-uniform).
-__device__ __forceinline__ void chunk_segments(const BlockParams& bp, int64_t chunk_unit0, int& s_lo, int& s_hi) {
-    const int64_t j_lo = chunk_unit0 << 2;
-    int64_t j_hi = j_lo + kChunkCoords;
+// Segment range [s_lo, s_hi] of the chunk that starts at unit `chunk_unit0` (warp-uniform): one load
+// from the table built when the partition was set; only a chunk that crosses a boundary searches.
+__device__ __forceinline__ int32_t chunk_entry(const BlockParams& bp, int64_t chunk_unit0) {
+    return __ldg(&bp.chunk_seg[chunk_unit0 >> 5]);
+}
+__device__ __forceinline__ void chunk_segments_from(const BlockParams& bp, int32_t entry, int64_t chunk_unit0, int& s_lo,
+                                                    int& s_hi) {
+    s_lo = entry & 0x7FFFFFFF;
+    s_hi = s_lo;
+    if (entry >= 0) return;
+    int64_t j_hi = (chunk_unit0 << 2) + kChunkCoords;
     if (j_hi > bp.covered_end) j_hi = bp.covered_end;
-    s_lo = seg_of(bp, j_lo);
-    s_hi = (j_hi - 1 < __ldg(&bp.offsets[s_lo + 1])) ? s_lo : seg_of(bp, j_hi - 1);
+    if (j_hi - 1 >= __ldg(&bp.offsets[s_lo + 1])) s_hi = seg_of(bp, j_hi - 1);
+}
+__device__ __forceinline__ void chunk_segments(const BlockParams& bp, int64_t chunk_unit0, int& s_lo, int& s_hi) {
+    chunk_segments_from(bp, chunk_entry(bp, chunk_unit0), chunk_unit0, s_lo, s_hi);
+}
+
+// Table of chunk_segments: entry k describes coordinates [128 k, min(128 k + 128, d)).
+__global__ void __launch_bounds__(256) chunk_table_kernel(const int64_t* offsets, int32_t B, int64_t d, int32_t* chunk_seg,
+                                                          int64_t chunks) {
+    const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= chunks) return;
+    BlockParams bp = {};
+    bp.offsets = offsets;
+    bp.B = B;
+    const int64_t j_lo = k * kChunkCoords;
+    int64_t j_hi = j_lo + kChunkCoords;
+    if (j_hi > d) j_hi = d;
+    const int s = seg_of(bp, j_lo);
+    const bool crosses = (j_hi - 1) >= offsets[s + 1];
+    chunk_seg[k] = s | (crosses ? (int32_t)0x80000000 : 0);
 }
 
 __device__ __forceinline__ UnitScale unit_scale(const BlockParams& bp, int64_t unit, int s_lo, int s_hi) {
@@ -111,6 +136,7 @@ struct BlockState {
     float* alpha;       // B
     float* c;           // B
     double* chunk_sum;
+    const int32_t* chunk_seg;
     double* edge_sum;
     double* tail_sq;
     int32_t B;

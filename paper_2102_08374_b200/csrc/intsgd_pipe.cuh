@@ -252,6 +252,21 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         uint32_t s = 0, phase = 0;
         float max_sum = 0.0f;                                            // max |S| over fast-path units
         const bool count_overflow = P.agg_limit != 0x7FFFFFFF;          // int8 wire: count |S| > 127
+        // Block-wise scales: the table entry of each of the thread's chunks and the scale of its first
+        // segment are fetched one tile ahead, so that no load sits between two tiles.
+        int32_t ent[UPT], ent_next[UPT];
+        float pre_a[UPT], pre_c[UPT];
+#pragma unroll
+        for (int k = 0; k < UPT; ++k) {
+            ent[k] = ent_next[k] = 0;
+            pre_a[k] = pre_c[k] = 0.0f;
+            if (BLOCKS) {
+                const int64_t chunk0 = (int64_t)blockIdx.x * kTileUnits + c + (int64_t)k * NC - lane;
+                if (chunk0 < PP.units) ent[k] = chunk_entry(bp, chunk0);
+                pre_a[k] = __ldg(&bp.alpha[ent[k] & 0x7FFFFFFF]);
+                pre_c[k] = __ldg(&bp.c[ent[k] & 0x7FFFFFFF]);
+            }
+        }
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             const int64_t unit0 = tile * kTileUnits + c;
             float4 xo[UPT];
@@ -259,6 +274,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
             UnitAcc ua[UPT];
             float2 a01[UPT], a23[UPT];
             int s_lo[UPT], s_hi[UPT];
+            float c_uni[UPT];
             bool active[UPT], half[UPT];
 #pragma unroll
             for (int k = 0; k < UPT; ++k) {
@@ -277,14 +293,23 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 a01[k] = make_float2(alpha, alpha);
                 a23[k] = a01[k];
                 s_lo[k] = s_hi[k] = 0;
+                c_uni[k] = 0.0f;
                 if (BLOCKS) {
                     // the warp's 32 units form one chunk; chunks past the covered range are never committed
-                    if (unit - lane < PP.units) chunk_segments(bp, unit - lane, s_lo[k], s_hi[k]);
+                    if (unit - lane < PP.units) chunk_segments_from(bp, ent[k], unit - lane, s_lo[k], s_hi[k]);
                     if (active[k]) {
-                        const UnitScale us = unit_scale(bp, unit, s_lo[k], s_hi[k]);
-                        a01[k] = us.a01;
-                        a23[k] = us.a23;
+                        if (s_lo[k] == s_hi[k]) {   // the chunk lies in one segment: scale and decode factor are at hand
+                            a01[k] = make_float2(pre_a[k], pre_a[k]);
+                            a23[k] = a01[k];
+                            c_uni[k] = pre_c[k];
+                        } else {
+                            const UnitScale us = unit_scale(bp, unit, s_lo[k], s_hi[k]);
+                            a01[k] = us.a01;
+                            a23[k] = us.a23;
+                        }
                     }
+                    const int64_t next_chunk0 = unit - lane + (int64_t)gridDim.x * kTileUnits;
+                    ent_next[k] = (next_chunk0 < PP.units) ? chunk_entry(bp, next_chunk0) : 0;
                 }
             }
             for (int g0 = 0; g0 < n; g0 += G) {
@@ -323,70 +348,96 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 if (++s == NS) { s = 0; phase ^= 1u; }
             }
             if (!ok) break;
+            float next_a[UPT], next_c[UPT];
+#pragma unroll
+            for (int k = 0; k < UPT; ++k) {
+                next_a[k] = next_c[k] = 0.0f;
+                if (BLOCKS) {   // the entries have arrived during the tile; these two loads overlap the epilogue
+                    next_a[k] = __ldg(&bp.alpha[ent_next[k] & 0x7FFFFFFF]);
+                    next_c[k] = __ldg(&bp.c[ent_next[k] & 0x7FFFFFFF]);
+                }
+            }
 #pragma unroll
             for (int k = 0; k < UPT; ++k) {
                 const int64_t unit = unit0 + (int64_t)k * NC;
                 if (BLOCKS) {
                     if (unit - lane >= PP.units) continue;   // warp-uniform: this chunk does not exist
-                    double sq[4] = {0.0, 0.0, 0.0, 0.0};
-                    int seg[4] = {-1, -1, -1, -1};
-                    if (active[k]) {
-                        const UnitScale us = unit_scale(bp, unit, s_lo[k], s_hi[k]);
-                        int4 S;
-                        float4 Sf;
-                        if (ua[k].m <= PP.fast_limit) {
-                            Sf = make_float4(ua[k].F01.x, ua[k].F01.y, ua[k].F23.x, ua[k].F23.y);
-                            S = make_int4(__float2int_rn(Sf.x), __float2int_rn(Sf.y), __float2int_rn(Sf.z), __float2int_rn(Sf.w));
-                        } else {
-                            S = redo_unit<GRAD, ROUND>(P, unit, make_float4(us.a01.x, us.a01.y, us.a23.x, us.a23.y), step, s_cnt);
-                            Sf = make_float4(__int2float_rn(S.x), __int2float_rn(S.y), __int2float_rn(S.z), __int2float_rn(S.w));
-                        }
-                        float4 xn;
-                        xn.x = update_coord_sq(xo[k].x, Sf.x, us.c.x, sq[0]);
-                        xn.y = update_coord_sq(xo[k].y, Sf.y, us.c.y, sq[1]);
-                        xn.z = update_coord_sq(xo[k].z, Sf.z, us.c.z, sq[2]);
-                        xn.w = update_coord_sq(xo[k].w, Sf.w, us.c.w, sq[3]);
-                        store_f4<true>(P.x, unit, xn);
-                        if (P.agg) store_i4<true>(P.agg, unit, S);
-                        note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
-                        note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
+                    if (s_lo[k] != s_hi[k]) {
+                        // the chunk crosses a segment boundary: per-coordinate scales, one partial per segment
+                        double sq[4] = {0.0, 0.0, 0.0, 0.0};
+                        int seg[4] = {-1, -1, -1, -1};
+                        if (active[k]) {
+                            const UnitScale us = unit_scale(bp, unit, s_lo[k], s_hi[k]);
+                            int4 S;
+                            if (ua[k].m <= PP.fast_limit)
+                                S = make_int4(__float2int_rn(ua[k].F01.x), __float2int_rn(ua[k].F01.y),
+                                              __float2int_rn(ua[k].F23.x), __float2int_rn(ua[k].F23.y));
+                            else
+                                S = redo_unit<GRAD, ROUND>(P, unit, make_float4(us.a01.x, us.a01.y, us.a23.x, us.a23.y), step, s_cnt);
+                            float4 xn;
+                            xn.x = update_coord_sq(xo[k].x, __int2float_rn(S.x), us.c.x, sq[0]);
+                            xn.y = update_coord_sq(xo[k].y, __int2float_rn(S.y), us.c.y, sq[1]);
+                            xn.z = update_coord_sq(xo[k].z, __int2float_rn(S.z), us.c.z, sq[2]);
+                            xn.w = update_coord_sq(xo[k].w, __int2float_rn(S.w), us.c.w, sq[3]);
+                            store_f4<true>(P.x, unit, xn);
+                            if (P.agg) store_i4<true>(P.agg, unit, S);
+                            note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
+                            note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
+                            for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
+                        }
+                        chunk_commit(bp, unit - lane, s_lo[k], s_hi[k], sq, seg);
+                        continue;
                     }
-                    chunk_commit(bp, unit - lane, s_lo[k], s_hi[k], sq, seg);
+                } else if (!active[k]) {
                     continue;
                 }
-                if (!active[k]) continue;
-                int4 S;
-                float2 S01, S23;   // the sums as floats (exact on the fast path)
-                if (ua[k].m <= PP.fast_limit) {
-                    S01 = ua[k].F01;
-                    S23 = ua[k].F23;
-                    S = make_int4(__float2int_rn(S01.x), __float2int_rn(S01.y), __float2int_rn(S23.x), __float2int_rn(S23.y));
-                    max_sum = absmax3_nan(max_sum, S01.x, S01.y);
-                    max_sum = absmax3_nan(max_sum, S23.x, S23.y);
-                    if (count_overflow)
-                        acc.overflow += (fabsf(S01.x) > 127.0f) + (fabsf(S01.y) > 127.0f) + (fabsf(S23.x) > 127.0f) +
-                                        (fabsf(S23.y) > 127.0f);
-                } else {
-                    S = redo_unit<GRAD, ROUND>(P, unit, make_float4(alpha, alpha, alpha, alpha), step, s_cnt);
-                    S01 = make_float2(__int2float_rn(S.x), __int2float_rn(S.y));
-                    S23 = make_float2(__int2float_rn(S.z), __int2float_rn(S.w));
-                    note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
-                    note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
+                // One scale for the whole unit (always, or a chunk inside one segment).
+                double unit_sq = 0.0;   // squared step of the unit: ((d0^2 + d1^2) + d2^2) + d3^2, products exact
+                if (active[k]) {
+                    const float cu = BLOCKS ? c_uni[k] : cdec;
+                    int4 S;
+                    float2 S01, S23;   // the sums as floats (exact on the fast path)
+                    if (ua[k].m <= PP.fast_limit) {
+                        S01 = ua[k].F01;
+                        S23 = ua[k].F23;
+                        S = make_int4(__float2int_rn(S01.x), __float2int_rn(S01.y), __float2int_rn(S23.x), __float2int_rn(S23.y));
+                        max_sum = absmax3_nan(max_sum, S01.x, S01.y);
+                        max_sum = absmax3_nan(max_sum, S23.x, S23.y);
+                        if (count_overflow)
+                            acc.overflow += (fabsf(S01.x) > 127.0f) + (fabsf(S01.y) > 127.0f) + (fabsf(S23.x) > 127.0f) +
+                                            (fabsf(S23.y) > 127.0f);
+                    } else {
+                        S = redo_unit<GRAD, ROUND>(P, unit, make_float4(a01[k].x, a01[k].y, a23[k].x, a23[k].y), step, s_cnt);
+                        S01 = make_float2(__int2float_rn(S.x), __int2float_rn(S.y));
+                        S23 = make_float2(__int2float_rn(S.z), __int2float_rn(S.w));
+                        note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
+                        note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
+                    }
+                    // t = fl(c S); x_new = fl(x - t); dj = fl(x_new - x): packed, each rounded once
+                    const float2 neg1 = make_float2(-1.0f, -1.0f), c2 = make_float2(cu, cu);
+                    const float2 xo01 = make_float2(xo[k].x, xo[k].y), xo23 = make_float2(xo[k].z, xo[k].w);
+                    const float2 xn01 = __ffma2_rn(__fmul2_rn(c2, S01), neg1, xo01);
+                    const float2 xn23 = __ffma2_rn(__fmul2_rn(c2, S23), neg1, xo23);
+                    const float2 d01 = __ffma2_rn(xo01, neg1, xn01), d23 = __ffma2_rn(xo23, neg1, xn23);
+                    double* sink = BLOCKS ? &unit_sq : &acc.dx2;
+                    *sink = __fma_rn((double)d01.x, (double)d01.x, *sink);
+                    *sink = __fma_rn((double)d01.y, (double)d01.y, *sink);
+                    *sink = __fma_rn((double)d23.x, (double)d23.x, *sink);
+                    *sink = __fma_rn((double)d23.y, (double)d23.y, *sink);
+                    store_f4<true>(P.x, unit, make_float4(xn01.x, xn01.y, xn23.x, xn23.y));
+                    if (P.agg) store_i4<true>(P.agg, unit, S);
                 }
-                // t = fl(c S); x_new = fl(x - t); dj = fl(x_new - x): packed, each rounded once
-                const float2 neg1 = make_float2(-1.0f, -1.0f), c2 = make_float2(cdec, cdec);
-                const float2 xo01 = make_float2(xo[k].x, xo[k].y), xo23 = make_float2(xo[k].z, xo[k].w);
-                const float2 xn01 = __ffma2_rn(__fmul2_rn(c2, S01), neg1, xo01);
-                const float2 xn23 = __ffma2_rn(__fmul2_rn(c2, S23), neg1, xo23);
-                const float2 d01 = __ffma2_rn(xo01, neg1, xn01), d23 = __ffma2_rn(xo23, neg1, xn23);
-                acc.dx2 = __fma_rn((double)d01.x, (double)d01.x, acc.dx2);
-                acc.dx2 = __fma_rn((double)d01.y, (double)d01.y, acc.dx2);
-                acc.dx2 = __fma_rn((double)d23.x, (double)d23.x, acc.dx2);
-                acc.dx2 = __fma_rn((double)d23.y, (double)d23.y, acc.dx2);
-                store_f4<true>(P.x, unit, make_float4(xn01.x, xn01.y, xn23.x, xn23.y));
-                if (P.agg) store_i4<true>(P.agg, unit, S);
+                if (BLOCKS) {   // all 32 lanes of the warp: one partial per chunk, fixed order
+                    const double t = warp_tree(unit_sq);
+                    if (lane == 0) __stcg(&bp.chunk_sum[(unit - lane) >> 5], t);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < UPT; ++k) {
+                ent[k] = ent_next[k];
+                pre_a[k] = next_a[k];
+                pre_c[k] = next_c[k];
             }
         }
         {   // fold the float-tracked maximum of the fast-path sums (integers below 2^24) into the counters
