@@ -4,9 +4,9 @@
 // keeps ~200 KB of loads in flight per SM independently of the consumers' register use, which is
 // what a 17-stream read at HBM3e speed needs.
 //
-// Layout of one stage: G worker tiles back to back, each kConsumers units of 16 (fp32) or 8 (bf16)
-// bytes; consumer thread c owns unit c of every tile, so shared-memory reads are conflict-free
-// 16-byte (8-byte) accesses and the Philox counter of a thread is fixed for a whole tile.
+// Layout of one stage: G worker tiles back to back, each NC * UPT units of 16 (fp32) or 8 (bf16)
+// bytes; consumer thread c owns units c, c + NC, ... of every tile, so shared-memory reads are
+// conflict-free 16-byte (8-byte) accesses and the Philox counters of a thread are fixed for a whole tile.
 //
 // Requirements checked by the host: every pointer 16-byte aligned, d <= 2^34.  Everything else
 // (unaligned pointers, larger d) runs in fused_step_kernel.
