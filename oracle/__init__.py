@@ -21,7 +21,7 @@ _LIB = _HERE / "liboracle_intsgd.so"
 
 GRAD_F32, GRAD_BF16 = 0, 1
 PAYLOAD_I32, PAYLOAD_I8 = 0, 1
-ROUND_RANDOM, ROUND_NEAREST, ROUND_RANDOM16 = 0, 1, 2
+ROUND_RANDOM, ROUND_NEAREST, ROUND_RANDOM16, ROUND_RANDOM_COMPARE = 0, 1, 2, 3
 INT32_MAX = 2**31 - 1
 
 
@@ -55,6 +55,10 @@ def _declare(L: C.CDLL) -> C.CDLL:
     L.orc_int_round.restype = C.c_int32
     L.orc_int_round_nearest.argtypes = [C.c_float]
     L.orc_int_round_nearest.restype = C.c_int32
+    L.orc_int_round_compare.argtypes = [C.c_float, C.c_float]
+    L.orc_int_round_compare.restype = C.c_int32
+    L.orc_uniform24_from_word.argtypes = [C.c_uint32]
+    L.orc_uniform24_from_word.restype = C.c_float
     L.orc_limit_as_float.argtypes = [C.c_int64]
     L.orc_limit_as_float.restype = C.c_float
     L.orc_scale.argtypes = [C.c_int64, C.c_int32, C.c_double, C.c_double, C.c_double,
@@ -141,6 +145,14 @@ def uniform_from_word(w: int) -> float:
 
 def int_round(y: float, u: float) -> int:
     return int(lib().orc_int_round(y, u))
+
+
+def int_round_compare(y: float, u: float) -> int:
+    return int(lib().orc_int_round_compare(y, u))
+
+
+def uniform24_from_word(w: int) -> float:
+    return float(lib().orc_uniform24_from_word(w))
 
 
 def int_round_nearest(y: float) -> int:

@@ -101,6 +101,11 @@ float uniform_from_word(uint32_t w) {
     return (float)w * 2.3283064365386963e-10f;           // 2^-32; at most 24 significant bits: exact
 }
 
+// 24-bit uniform in [0, 1) of rounding mode 3: the top 24 bits of the word times 2^-24; exact in fp32.
+float uniform24_from_word(uint32_t w) {
+    return (float)(w >> 8) * 5.9604644775390625e-8f;  // 2^-24
+}
+
 float widen_bf16(uint16_t h) {
     const uint32_t bits = (uint32_t)h << 16;
     float f;
@@ -134,6 +139,15 @@ float int_round_random(float y, float u) {
     return ((double)u >= need) ? (float)((double)k + 1.0) : k;
 }
 
+// The same Int(t) drawn by comparison (rounding mode 3): floor(t) + 1 iff u < p with
+// p = fl32(t - floor(t)), the fractional part as fp32 arithmetic gives it (rounded only for
+// -1 < t < 0 with bits below 2^-24, where fl32(t + 1) can reach 1).
+float int_round_random_compare(float y, float u) {
+    const float f = std::floor(y);
+    const float p = y - f;
+    return f + ((u < p) ? 1.0f : 0.0f);
+}
+
 // Deterministic variant named in Section 5.1 ("IntSGD (Determ.)"): round to nearest, ties
 // to even.
 float int_round_nearest(float y) {
@@ -146,7 +160,10 @@ struct Rounded { int32_t q; bool clipped; bool nonfinite; };
 
 Rounded round_and_clip(float y, float u, float Lf, int rounding) {
     Rounded r;
-    float qf = (rounding == 1) ? int_round_nearest(y) : int_round_random(y, u);
+    float qf;
+    if (rounding == 1) qf = int_round_nearest(y);
+    else if (rounding == 3) qf = int_round_random_compare(y, u);
+    else qf = int_round_random(y, u);
     r.clipped = !(std::fabs(y) <= Lf);
     r.nonfinite = !std::isfinite(y);
     if (y > Lf) qf = Lf;
@@ -175,6 +192,8 @@ float orc_draw_uniform16(uint64_t seed, uint32_t step, uint32_t worker, uint64_t
 // ---- Int(t), Section 2 ------------------------------------------------------------------
 int32_t orc_int_round(float y, float u) { return (int32_t)int_round_random(y, u); }
 int32_t orc_int_round_nearest(float y) { return (int32_t)int_round_nearest(y); }
+int32_t orc_int_round_compare(float y, float u) { return (int32_t)int_round_random_compare(y, u); }
+float orc_uniform24_from_word(uint32_t w) { return uniform24_from_word(w); }
 float orc_limit_as_float(int64_t L) { return limit_as_float(L); }
 
 // ---- Algorithm 1, the two scalar lines: moving average r_k and scale alpha_k ------------
@@ -225,7 +244,7 @@ void orc_scale_block(int64_t d, int64_t d_l, int32_t n, double eta, double beta,
 // One worker, coordinates [j0, j0 + count) of a vector whose element 0 is grad[0]
 // (grad, payload and u_inject are indexed relative to j0; the random stream by j0 + t).
 // grad_dtype 0 = fp32, 1 = bf16; payload_dtype 0 = int32, 1 = int8; rounding 0 = random (one Philox word per draw),
-// 2 = random with the 16-bit draws of draw_uniform16,
+// 2 = random with the 16-bit draws of draw_uniform16, 3 = random by comparison with a 24-bit draw,
 // 1 = nearest-even.  u_inject (nullable) replaces the Philox draw, for hand examples.
 void orc_encode(const void* grad, int grad_dtype, int64_t j0, int64_t count, float alpha,
                 int64_t L, int payload_dtype, int rounding, uint64_t seed, uint32_t step,
@@ -239,6 +258,7 @@ void orc_encode(const void* grad, int grad_dtype, int64_t j0, int64_t count, flo
         if (rounding != 1) {
             if (u_inject) u = u_inject[t];
             else if (rounding == 2) u = draw_uniform16(seed, step, worker, (uint64_t)(j0 + t));
+            else if (rounding == 3) u = uniform24_from_word(draw_word(seed, step, worker, (uint64_t)(j0 + t)));
             else u = uniform_from_word(draw_word(seed, step, worker, (uint64_t)(j0 + t)));
         }
         const Rounded r = round_and_clip(y, u, Lf, rounding);
@@ -361,6 +381,7 @@ void orc_diana_step_window(const void* const* grads, int grad_dtype, int32_t n, 
             const float y = alpha * v;
             float u = 0.0f;
             if (rounding == 2) u = draw_uniform16(seed, step, (uint32_t)i, (uint64_t)(j0 + t));
+            else if (rounding == 3) u = uniform24_from_word(draw_word(seed, step, (uint32_t)i, (uint64_t)(j0 + t)));
             else if (rounding == 0) u = uniform_from_word(draw_word(seed, step, (uint32_t)i, (uint64_t)(j0 + t)));
             const Rounded r = round_and_clip(y, u, Lf, rounding);
             if (r.clipped) clip_count[i] += 1;

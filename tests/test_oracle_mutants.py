@@ -8,6 +8,7 @@ import pytest
 
 import oracle
 import test_oracle_blocks as tb
+import test_oracle_compare as tc
 import test_oracle_diana as td
 import test_oracle_draw16 as t16
 import test_oracle_heuristic as th
@@ -34,6 +35,9 @@ MUTANTS = [
     ("draw: complement dropped", "const double need = ((double)k + 1.0) - (double)y;", "const double need = (double)y - (double)k;"),
     ("draw: sum rounded to fp32 before the floor", "return ((double)u >= need) ? (float)((double)k + 1.0) : k;", "return std::floor(y + u);"),
     ("floor replaced by truncation", "const float k = std::floor(y);", "const float k = std::trunc(y);"),
+    ("compare form: up iff u <= p", "return f + ((u < p) ? 1.0f : 0.0f);", "return f + ((u <= p) ? 1.0f : 0.0f);"),
+    ("compare form: 23-bit draw", "return (float)(w >> 8) * 5.9604644775390625e-8f;", "return (float)(w >> 9) * 5.9604644775390625e-8f;"),
+    ("compare form: truncation for floor", "const float f = std::floor(y);", "const float f = std::trunc(y);"),
     ("nearest: ties away from zero", "return std::nearbyintf(y);", "return std::roundf(y);"),
     ("clip: NaN not zeroed", "    if (y != y) qf = 0.0f;\n", ""),
     ("clip: limit off by one", "if (y > Lf) qf = Lf;", "if (y > Lf) qf = Lf + 1.0f;"),
@@ -100,6 +104,9 @@ def _battery():
     td.test_zero_shifts_give_the_intsgd_integers_and_step()
     th.test_hand_values()
     t16.test_layout_against_an_independent_statement()
+    tc.test_uniform24_is_the_top_24_bits()
+    tc.test_definition_against_exact_rationals()
+    tc.test_half_integers_and_boundaries()
 
 
 def test_the_unmodified_oracle_passes_the_battery(tmp_path, monkeypatch):
