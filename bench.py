@@ -67,8 +67,9 @@ def parse_args():
     p.add_argument("--payload", default="int32", choices=["int32", "int8"])
     p.add_argument("--grad", default="f32", choices=["f32", "bf16"])
     p.add_argument("--mode", default="fused", choices=["fused", "two_kernel"])
-    p.add_argument("--rounding", default="random", choices=["random", "nearest", "random16"],
-                   help="random16 = the optional 16-bit draw stream (a different random stream; not the default)")
+    p.add_argument("--rounding", default="random", choices=["random", "nearest", "random16", "compare"],
+                   help="random16 = the optional 16-bit draw stream; compare = Int(t) drawn by comparing a 24-bit "
+                        "uniform with the fractional part (both: a different random stream; not the default)")
     p.add_argument("--eta", type=float, default=0.1)
     p.add_argument("--e2e-steps", type=int, default=3)
     p.add_argument("--cpu-sample-log2", type=int, default=24,
@@ -163,7 +164,7 @@ def oracle_sample_throughput(n, d, sample_log2, grad_dtype, payload, rounding, s
         grads = [synth.to_bf16_bits(g) for g in grads]
     x = synth.iterate(w)
     pd = oracle.PAYLOAD_I8 if payload == "int8" else oracle.PAYLOAD_I32
-    rd = {"nearest": oracle.ROUND_NEAREST, "random16": oracle.ROUND_RANDOM16}.get(rounding, oracle.ROUND_RANDOM)
+    rd = {"nearest": oracle.ROUND_NEAREST, "random16": oracle.ROUND_RANDOM16, "compare": oracle.ROUND_RANDOM_COMPARE}.get(rounding, oracle.ROUND_RANDOM)
     oracle.step_window([g[:1024] for g in grads], x[:1024].copy(), np.float32(700.0), np.float32(1e-5), step=1,
                        seed=seed, payload_dtype=pd, rounding=rd)     # load the library, touch the code
     t = time.perf_counter()
@@ -233,7 +234,7 @@ def main():
     n, d = args.workers, 1 << args.log2d
     grad_dtype = pkg.GRAD_BF16 if args.grad == "bf16" else pkg.GRAD_F32
     payload_dtype = pkg.PAYLOAD_I8 if args.payload == "int8" else pkg.PAYLOAD_I32
-    rounding = {"nearest": pkg.ROUND_NEAREST, "random16": pkg.ROUND_RANDOM16}.get(args.rounding, pkg.ROUND_RANDOM)
+    rounding = {"nearest": pkg.ROUND_NEAREST, "random16": pkg.ROUND_RANDOM16, "compare": pkg.ROUND_RANDOM_COMPARE}.get(args.rounding, pkg.ROUND_RANDOM)
     mode = pkg.MODE_TWO_KERNEL if args.mode == "two_kernel" else pkg.MODE_FUSED
     gb, pb = (2 if args.grad == "bf16" else 4), (1 if args.payload == "int8" else 4)
 

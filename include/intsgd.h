@@ -68,6 +68,9 @@ extern "C" {
                                     e = j mod 4 uses the low (e even) or high (e odd) 16 bits v of word
                                     2h + e / 2; Int(y) = floor(y + v * 2^-16).  Bias at most
                                     2^-16 per value.  Halves the random-number work: an option, not the default */
+#define INTSGD_ROUND_RANDOM_COMPARE 3  /* Int(t) drawn by comparison: u = (word >> 8) * 2^-24 (24 bits), up iff
+                                          u < fl32(y - floor(y)).  Same law and same Philox words as
+                                          INTSGD_ROUND_RANDOM, different draws; three more instructions per value */
 #define INTSGD_MODE_EXACT      0 /* Algorithm 1, Init line: x <- x - eta (1/n) sum_i g_i, uncompressed */
 #define INTSGD_MODE_TWO_KERNEL 1 /* encode every worker to a payload buffer, then aggregate */
 #define INTSGD_MODE_FUSED      2 /* one pass, payloads never reach memory */

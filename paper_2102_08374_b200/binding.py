@@ -26,7 +26,7 @@ NOALLOC_MAX_D = 1 << 28
 
 GRAD_F32, GRAD_BF16 = 0, 1
 PAYLOAD_I32, PAYLOAD_I8 = 0, 1
-ROUND_RANDOM, ROUND_NEAREST, ROUND_RANDOM16 = 0, 1, 2
+ROUND_RANDOM, ROUND_NEAREST, ROUND_RANDOM16, ROUND_RANDOM_COMPARE = 0, 1, 2, 3
 MODE_EXACT, MODE_TWO_KERNEL, MODE_FUSED = 0, 1, 2
 
 EXPORTS = [

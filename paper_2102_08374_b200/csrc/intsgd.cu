@@ -179,6 +179,8 @@ void launch_encode_r(const intsgd_ctx* ctx, const VecParams& P, dim3 grid, cudaS
         encode_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
     else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM16)
         encode_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_RANDOM16><<<grid, ctx->threads, 0, s>>>(P);
+    else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM_COMPARE)
+        encode_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_RANDOM_COMPARE><<<grid, ctx->threads, 0, s>>>(P);
     else
         encode_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
@@ -220,6 +222,8 @@ void launch_fused_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStr
         fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
     else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM16)
         fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM16><<<grid, ctx->threads, 0, s>>>(P);
+    else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM_COMPARE)
+        fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM_COMPARE><<<grid, ctx->threads, 0, s>>>(P);
     else
         fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
@@ -305,9 +309,11 @@ int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     cudaError_t e;
     if (!bf16 && rounding == INTSGD_ROUND_RANDOM) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_RANDOM>(ctx, PP, s);
     else if (!bf16 && rounding == INTSGD_ROUND_RANDOM16) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_RANDOM16>(ctx, PP, s);
+    else if (!bf16 && rounding == INTSGD_ROUND_RANDOM_COMPARE) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_RANDOM_COMPARE>(ctx, PP, s);
     else if (!bf16) e = launch_pipe_t<INTSGD_GRAD_F32, INTSGD_ROUND_NEAREST>(ctx, PP, s);
     else if (rounding == INTSGD_ROUND_RANDOM) e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_RANDOM>(ctx, PP, s);
     else if (rounding == INTSGD_ROUND_RANDOM16) e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_RANDOM16>(ctx, PP, s);
+    else if (rounding == INTSGD_ROUND_RANDOM_COMPARE) e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_RANDOM_COMPARE>(ctx, PP, s);
     else e = launch_pipe_t<INTSGD_GRAD_BF16, INTSGD_ROUND_NEAREST>(ctx, PP, s);
     if (e != cudaSuccess) {
         std::snprintf(ctx->err, 256, "fused_pipe_kernel setup failed: %s", cudaGetErrorString(e));
@@ -324,6 +330,8 @@ void launch_fused_blocks_r(const intsgd_ctx* ctx, const VecParams& P, int grid, 
         fused_step_blocks_kernel<GRAD, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
     else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM16)
         fused_step_blocks_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM16><<<grid, ctx->threads, 0, s>>>(P);
+    else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM_COMPARE)
+        fused_step_blocks_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM_COMPARE><<<grid, ctx->threads, 0, s>>>(P);
     else
         fused_step_blocks_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
@@ -358,6 +366,8 @@ void launch_diana_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStr
         diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P);
     else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM16)
         diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM16><<<grid, ctx->threads, 0, s>>>(P);
+    else if (ctx->cfg.rounding == INTSGD_ROUND_RANDOM_COMPARE)
+        diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM_COMPARE><<<grid, ctx->threads, 0, s>>>(P);
     else
         diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
@@ -494,7 +504,7 @@ int intsgd_create(intsgd_ctx** out, const intsgd_config* cfg) {
     if (cfg->payload_dtype != INTSGD_PAYLOAD_I32 && cfg->payload_dtype != INTSGD_PAYLOAD_I8)
         return fail(nullptr, INTSGD_ERR_INVALID_ARG, "bad payload_dtype");
     if (cfg->rounding != INTSGD_ROUND_RANDOM && cfg->rounding != INTSGD_ROUND_NEAREST &&
-        cfg->rounding != INTSGD_ROUND_RANDOM16)
+        cfg->rounding != INTSGD_ROUND_RANDOM16 && cfg->rounding != INTSGD_ROUND_RANDOM_COMPARE)
         return fail(nullptr, INTSGD_ERR_INVALID_ARG, "bad rounding");
     if (!(cfg->beta >= 0.0 && cfg->beta < 1.0)) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "beta must be in [0, 1)");
     if (!(cfg->eps >= 0.0) || !std::isfinite(cfg->eps)) return fail(nullptr, INTSGD_ERR_INVALID_ARG, "eps must be finite and >= 0");

@@ -130,14 +130,26 @@ __device__ __forceinline__ uint4 draw_unit(int64_t unit, uint32_t worker, uint32
 }
 
 // The uniform draw is draw_as_float(w) * draw_scale(): the word times 2^-32 truncated to fp32 (the
-// conversion rounds toward zero, so u <= 1 - 2^-24), or the 16-bit value times 2^-16.
+// conversion rounds toward zero, so u <= 1 - 2^-24), the 16-bit value times 2^-16, or (compare form)
+// the word's top 24 bits times 2^-24.
 template <int ROUND>
 __device__ __forceinline__ float draw_as_float(uint32_t w) {
-    return (ROUND == INTSGD_ROUND_RANDOM16) ? __uint2float_rn(w) : __uint2float_rz(w);
+    if (ROUND == INTSGD_ROUND_RANDOM16) return __uint2float_rn(w);
+    if (ROUND == INTSGD_ROUND_RANDOM_COMPARE) return __uint2float_rn(w >> 8);
+    return __uint2float_rz(w);
 }
 template <int ROUND>
 __device__ __forceinline__ float draw_scale() {
-    return (ROUND == INTSGD_ROUND_RANDOM16) ? 1.52587890625e-05f : 2.3283064365386963e-10f;
+    if (ROUND == INTSGD_ROUND_RANDOM16) return 1.52587890625e-05f;
+    if (ROUND == INTSGD_ROUND_RANDOM_COMPARE) return 5.9604644775390625e-08f;
+    return 2.3283064365386963e-10f;
+}
+
+// 1.0f if a < b else 0.0f, in one instruction.
+__device__ __forceinline__ float lt_as_float(float a, float b) {
+    float d;
+    asm("set.lt.f32.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
 }
 
 // ----------------------------------------------------------------------------------------
@@ -212,6 +224,12 @@ __device__ __forceinline__ float absmax3_nan(float a, float b, float c) {
 template <int ROUND>
 __device__ __forceinline__ int round_in_range(float y, uint32_t w) {
     if (ROUND == INTSGD_ROUND_NEAREST) return __float2int_rn(y);
+    if (ROUND == INTSGD_ROUND_RANDOM_COMPARE) {
+        // compare form: f = floor(y), p = fl32(y - f), up iff u < p; done as (float)(w >> 8) < p * 2^24 (exact scalings)
+        const float f = floorf(y);
+        const float p = __fsub_rn(y, f);
+        return __float2int_rz(f) + (draw_as_float<ROUND>(w) < __fmul_rn(p, 16777216.0f) ? 1 : 0);
+    }
     return __float2int_rd(__fmaf_rd(draw_as_float<ROUND>(w), draw_scale<ROUND>(), y));
 }
 
@@ -256,6 +274,9 @@ template <int ROUND>
 __device__ __forceinline__ int4 round4_in_range(float2 y01, float2 y23, uint4 w) {
     if (ROUND == INTSGD_ROUND_NEAREST)
         return make_int4(__float2int_rn(y01.x), __float2int_rn(y01.y), __float2int_rn(y23.x), __float2int_rn(y23.y));
+    if (ROUND == INTSGD_ROUND_RANDOM_COMPARE)
+        return make_int4(round_in_range<ROUND>(y01.x, w.x), round_in_range<ROUND>(y01.y, w.y),
+                         round_in_range<ROUND>(y23.x, w.z), round_in_range<ROUND>(y23.y, w.w));
     const float2 scale = make_float2(draw_scale<ROUND>(), draw_scale<ROUND>());
     const float2 z01 = __ffma2_rd(make_float2(draw_as_float<ROUND>(w.x), draw_as_float<ROUND>(w.y)), scale, y01);
     const float2 z23 = __ffma2_rd(make_float2(draw_as_float<ROUND>(w.z), draw_as_float<ROUND>(w.w)), scale, y23);

@@ -78,6 +78,19 @@ __device__ __forceinline__ void consume_unit(float4 g, float2 alpha01, float2 al
         u.F23 = __fadd2_rn(u.F23, make_float2(rintf(y23.x), rintf(y23.y)));
         return;
     }
+    if (ROUND == INTSGD_ROUND_RANDOM_COMPARE) {
+        // f = floor(y); p = fl32(y - f); up iff (float)(w >> 8) < p * 2^24; every step rounded once
+        const float2 f01 = make_float2(floorf(y01.x), floorf(y01.y));
+        const float2 f23 = make_float2(floorf(y23.x), floorf(y23.y));
+        const float2 neg1 = make_float2(-1.0f, -1.0f), two24 = make_float2(16777216.0f, 16777216.0f);
+        const float2 p01 = __fmul2_rn(__ffma2_rn(f01, neg1, y01), two24);
+        const float2 p23 = __fmul2_rn(__ffma2_rn(f23, neg1, y23), two24);
+        const float2 u01 = make_float2(lt_as_float(draw_as_float<ROUND>(w.x), p01.x), lt_as_float(draw_as_float<ROUND>(w.y), p01.y));
+        const float2 u23 = make_float2(lt_as_float(draw_as_float<ROUND>(w.z), p23.x), lt_as_float(draw_as_float<ROUND>(w.w), p23.y));
+        u.F01 = __fadd2_rn(__fadd2_rn(u.F01, f01), u01);
+        u.F23 = __fadd2_rn(__fadd2_rn(u.F23, f23), u23);
+        return;
+    }
     // floor(y + u) on the unrounded sum: fused multiply-add rounded down, then floor (see round_in_range)
     const float2 scale = make_float2(draw_scale<ROUND>(), draw_scale<ROUND>());
     const float2 z01 = __ffma2_rd(make_float2(draw_as_float<ROUND>(w.x), draw_as_float<ROUND>(w.y)), scale, y01);
@@ -241,7 +254,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         const uint32_t step = st->step;
         const BlockParams& bp = P.bp;
         auto unit_draws = [&](const PhiloxThreadPart& t, const uint4& e, const uint4& pw, int k, bool h) -> uint4 {
-            if (ROUND == INTSGD_ROUND_RANDOM) return philox_finish(t, e, P.keys);
+            if (ROUND == INTSGD_ROUND_RANDOM || ROUND == INTSGD_ROUND_RANDOM_COMPARE) return philox_finish(t, e, P.keys);
             if (ROUND == INTSGD_ROUND_RANDOM16) {
                 if (kPairShared) return k == 0 ? split16(pw.x, pw.y) : split16(pw.z, pw.w);
                 const uint4 r = philox_finish(t, e, P.keys);
@@ -284,7 +297,8 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 xo[k] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (active[k]) xo[k] = load_f4<true>(P.x, unit);
                 tp[k].n3 = tp[k].H = tp[k].m1 = 0;
-                if (ROUND == INTSGD_ROUND_RANDOM) tp[k] = philox_thread_part((uint32_t)(unit + P.unit_base), step, P.keys);
+                if (ROUND == INTSGD_ROUND_RANDOM || ROUND == INTSGD_ROUND_RANDOM_COMPARE)
+                    tp[k] = philox_thread_part((uint32_t)(unit + P.unit_base), step, P.keys);
                 if (ROUND == INTSGD_ROUND_RANDOM16 && !(kPairShared && k > 0))
                     tp[k] = philox_thread_part(pair_index((uint32_t)(unit + P.unit_base)), step, P.keys);
                 ua[k].F01 = make_float2(0.f, 0.f);

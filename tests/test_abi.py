@@ -40,7 +40,7 @@ def test_argument_errors_need_no_gpu():
     assert b"NULL" in lib.intsgd_last_error(None)
     ctx = ctypes.c_void_p()
     from paper_2102_08374_b200.binding import Config
-    bad = [dict(n=0), dict(n=65), dict(d=0), dict(grad_dtype=7), dict(payload_dtype=3), dict(rounding=3), dict(rounding=-1),
+    bad = [dict(n=0), dict(n=65), dict(d=0), dict(grad_dtype=7), dict(payload_dtype=3), dict(rounding=4), dict(rounding=-1),
            dict(beta=1.0), dict(beta=-0.1), dict(eps=-1.0), dict(clip_limit=-5), dict(reserved=1),
            dict(payload_dtype=1, clip_limit=128), dict(n=16, clip_limit=2**28)]
     for kw in bad:

@@ -79,7 +79,7 @@ def _random_offsets(rng, d, B):
 @pytest.mark.parametrize("path,unaligned", [(0, False), (1, False), (1, True)])
 @pytest.mark.parametrize("grad_dtype,payload_dtype,rounding", [
     (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM), (pkg.GRAD_BF16, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM),
-    (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_NEAREST), (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM16)])
+    (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_NEAREST), (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM16), (pkg.GRAD_BF16, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM_COMPARE)])
 def test_blockwise_lockstep_with_ragged_segments(path, unaligned, grad_dtype, payload_dtype, rounding):
     """Segments of 1 to ~100k coordinates whose boundaries are not multiples of 4 or 128, a ragged
     tail, per-segment gradient scales spread over three decades."""

@@ -60,7 +60,7 @@ class DianaLockStep:
 @pytest.mark.parametrize("unaligned", [False, True])
 @pytest.mark.parametrize("grad_dtype,payload_dtype,rounding", [
     (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM), (pkg.GRAD_BF16, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM),
-    (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_NEAREST), (pkg.GRAD_BF16, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM16)])
+    (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_NEAREST), (pkg.GRAD_BF16, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM16), (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM_COMPARE)])
 def test_diana_lockstep_on_heterogeneous_quadratics(unaligned, grad_dtype, payload_dtype, rounding):
     """f_i(x) = |x - b_i|^2 / 2 with different b_i (heterogeneous data), full local gradients computed
     by the harness from the library's own iterate; several tiles and a ragged tail."""

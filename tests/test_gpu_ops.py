@@ -73,7 +73,7 @@ def test_sqdiff(d):
 
 @pytest.mark.parametrize("grad_dtype", [pkg.GRAD_F32, pkg.GRAD_BF16])
 @pytest.mark.parametrize("payload_dtype", [pkg.PAYLOAD_I32, pkg.PAYLOAD_I8])
-@pytest.mark.parametrize("rounding", [pkg.ROUND_RANDOM, pkg.ROUND_NEAREST, pkg.ROUND_RANDOM16])
+@pytest.mark.parametrize("rounding", [pkg.ROUND_RANDOM, pkg.ROUND_NEAREST, pkg.ROUND_RANDOM16, pkg.ROUND_RANDOM_COMPARE])
 def test_encode_bit_exact(grad_dtype, payload_dtype, rounding):
     rng = np.random.default_rng(11)
     n, seed = 5, 0xDEADBEEFCAFE

@@ -22,7 +22,7 @@ def _mode_and_path(which):
 @pytest.mark.parametrize("which", [FUSED_PIPELINED, FUSED_DIRECT, TWO_KERNEL])
 @pytest.mark.parametrize("grad_dtype,payload_dtype", [(pkg.GRAD_F32, pkg.PAYLOAD_I32), (pkg.GRAD_F32, pkg.PAYLOAD_I8),
                                                       (pkg.GRAD_BF16, pkg.PAYLOAD_I8), (pkg.GRAD_BF16, pkg.PAYLOAD_I32)])
-@pytest.mark.parametrize("rounding", [pkg.ROUND_RANDOM, pkg.ROUND_NEAREST, pkg.ROUND_RANDOM16])
+@pytest.mark.parametrize("rounding", [pkg.ROUND_RANDOM, pkg.ROUND_NEAREST, pkg.ROUND_RANDOM16, pkg.ROUND_RANDOM_COMPARE])
 def test_multi_step_lockstep(which, grad_dtype, payload_dtype, rounding):
     """Several tiles and a ragged tail: d = 5 * 2^16 + 3 spans many blocks and leaves 3 coordinates."""
     n, d, eta = 6, 5 * (1 << 16) + 3, 0.1
@@ -70,7 +70,8 @@ def test_two_kernel_payloads_match_the_oracle():
 @pytest.mark.parametrize("grad_dtype,payload_dtype,rounding", [
     (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM), (pkg.GRAD_BF16, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM),
     (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_NEAREST), (pkg.GRAD_BF16, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM),
-    (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM16), (pkg.GRAD_BF16, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM16)])
+    (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM16), (pkg.GRAD_BF16, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM16),
+    (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM_COMPARE)])
 def test_values_outside_the_fast_range_clip_and_count_exactly(which, grad_dtype, payload_dtype, rounding):
     """Huge, infinite and NaN gradients, and values between the fast-path range and the clip limit."""
     n, d, eta, seed = 5, 3 * 4096 + 9, 0.1, 77
@@ -104,7 +105,7 @@ def test_values_outside_the_fast_range_clip_and_count_exactly(which, grad_dtype,
 
 
 @pytest.mark.parametrize("which", [FUSED_PIPELINED, FUSED_DIRECT, TWO_KERNEL])
-@pytest.mark.parametrize("rounding", [pkg.ROUND_RANDOM, pkg.ROUND_RANDOM16])
+@pytest.mark.parametrize("rounding", [pkg.ROUND_RANDOM, pkg.ROUND_RANDOM16, pkg.ROUND_RANDOM_COMPARE])
 def test_values_next_to_integers_and_tiny_values(which, rounding):
     """Int(y) = floor(y + u) must be taken on the unrounded sum: scaled gradients a few ulps from an
     integer (both sides), exact integers, halves, and values down to the subnormals."""
