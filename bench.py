@@ -33,8 +33,8 @@ HBM_FALLBACK_GBS = 6650.0
 # command and figures in profiles/fused_pipe_kernel_d24_n16_ncu_full.md): bytes per coordinate of the
 # captured case (d = 2^24, n = 16, fp32, int32 aggregate), valid for the kernel sources with this hash.
 # Any change to the kernel sources makes `roofline.traffic` null until the counters are taken again.
-NCU_TRAFFIC = {"sources_sha256": "398ec93cee829894ff001ee38c4035fbbff4e7ab432ac913cba4763b3fa1121f",
-               "bytes_per_coordinate": 1.265483e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
+NCU_TRAFFIC = {"sources_sha256": "89ae7eff1f9a109b067b14ffa26f3e1847d8a5b8e41127d99d9d9ac78462f68a",
+               "bytes_per_coordinate": 1.265289e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
 
 
 def kernel_sources_hash():
@@ -76,6 +76,7 @@ def parse_args():
                    help="coordinates of the oracle sample (all workers), as a power of two")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
+    p.add_argument("--no-variants", action="store_true", help="skip the short runs of the other rounding modes")
     p.add_argument("--threads", type=int, default=0)
     p.add_argument("--blocks-per-sm", type=int, default=0)
     return p.parse_args()
@@ -296,6 +297,29 @@ def main():
                 "kernel_ms_median": statistics.median(per_step_ms),
                 "note": "per-step CUDA-event time (one-thread scale kernel + the vector kernel(s))"}
 
+    # ---- the other rounding modes on the same buffers, short bursts (context for the headline; 1 GPU only) ----
+    variants = None
+    if world == 1 and not args.no_variants and mode == pkg.MODE_FUSED:
+        variants = []
+        names = {"random": pkg.ROUND_RANDOM, "compare": pkg.ROUND_RANDOM_COMPARE, "random16": pkg.ROUND_RANDOM16,
+                 "nearest": pkg.ROUND_NEAREST}
+        for name, rd in names.items():
+            with pkg.IntSGD(n, d, grad_dtype=grad_dtype, payload_dtype=payload_dtype, rounding=rd, seed=1, device=local_rank) as vlib:
+                vlib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=pkg.MODE_EXACT, stream=stream)
+                for _ in range(3):
+                    vlib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=mode, stream=stream)
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(31)]
+                torch.cuda.synchronize()
+                ev[0].record()
+                for k in range(30):
+                    vlib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=mode, stream=stream)
+                    ev[k + 1].record()
+                torch.cuda.synchronize()
+                ms = statistics.median(ev[k].elapsed_time(ev[k + 1]) for k in range(30))
+            variants.append({"rounding": name, "burst_ms_median_of_30": ms,
+                             "hbm_frac": bytes_per_launch / (ms * 1e-3) / 1e9 / peak})
+            time.sleep(0.5)
+
     # ---- end to end through the host-buffer entry point (rank-local; max over ranks) ----
     e2e = None
     if not args.no_e2e and mode == pkg.MODE_FUSED:
@@ -332,7 +356,7 @@ def main():
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if args.grad == "f32" else "bf16->f32", "data": "synthetic", "config": workload_config(args),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-            "hbm_gbs_algorithmic": achieved * world,
+            "hbm_gbs_algorithmic": achieved * world, "rounding_variants": variants,
             "state": {"alpha": st["alpha"], "r": st["r"], "max_abs_agg": st["max_abs_agg"],
                       "clipped": sum(st["clip_count"]), "step": st["step"]},
         }
