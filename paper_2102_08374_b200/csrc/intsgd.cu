@@ -38,6 +38,7 @@ struct intsgd_ctx {
     void* stage_grads[INTSGD_MAX_WORKERS];
     float* stage_x;
     int32_t* stage_agg;
+    bool follows_scale;         // the next vector launch comes directly behind this step's scale kernel
     cudaStream_t back_stream;   // device->host copies of finished windows (non-blocking stream)
     cudaEvent_t window_done;
     char err[256];
@@ -47,6 +48,7 @@ namespace {
 
 thread_local char g_create_err[256] = "";
 
+constexpr int kMaxDevices = 64;
 constexpr int kDefaultThreads = 256;
 constexpr int kDefaultBlocksPerSm = 8;
 constexpr int kMaxBlocksPerSm = 32;
@@ -245,12 +247,28 @@ cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s)
     auto kernel = fused_pipe_kernel<GRAD, ROUND, BLOCKS, S.nc, S.upt, S.g, S.ns>;
     const int unit_bytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
     const int smem = S.ns * S.g * S.nc * S.upt * unit_bytes;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
+    static bool configured[kMaxDevices] = {};   // per instantiation and device: the opt-in to large shared memory
+    const int dev = ctx->cfg.device;
+    if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+    }
     PP.tiles = (PP.units + S.nc * S.upt - 1) / (S.nc * S.upt);
     int64_t grid = PP.tiles < ctx->sm_count ? PP.tiles : ctx->sm_count;
-    kernel<<<(unsigned)grid, S.nc + 32, smem, s>>>(PP);
-    return cudaSuccess;
+    // Launched right behind the step's scale kernel, the kernel may start while that one drains: it sets up
+    // its barriers and tables, then waits for the scale kernel's results (griddepcontrol.wait).
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(S.nc + 32, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->follows_scale ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, PP);
 }
 template <int GRAD, int ROUND>
 cudaError_t launch_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
@@ -674,7 +692,10 @@ int intsgd_step(intsgd_ctx* ctx, const void* const* grads, void* const* payload_
     }
     if (mode == INTSGD_MODE_FUSED) {
         if ((rc = launch_scale(ctx, eta_k, -1.0, s)) != INTSGD_OK) return rc;
-        return launch_fused(ctx, P, al, s);
+        ctx->follows_scale = true;
+        rc = launch_fused(ctx, P, al, s);
+        ctx->follows_scale = false;
+        return rc;
     }
     // TWO_KERNEL: the payload buffers' alignment decides the encode stores and aggregate loads.
     bool al_enc = al, al_agg = true;

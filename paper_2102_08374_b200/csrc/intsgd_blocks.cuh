@@ -149,6 +149,7 @@ struct BlockState {
 __global__ void __launch_bounds__(1024) scale_blocks_kernel(DevState* st, BlockState bs, double d_total, double two_n,
                                                             double n_as_double, double eta, double beta, double eps,
                                                             int32_t n) {
+    asm volatile("griddepcontrol.launch_dependents;");   // see scale_kernel
     int bad = 0;
     for (int l = threadIdx.x; l < bs.B; l += blockDim.x) {
         const double dl = (double)(bs.offsets[l + 1] - bs.offsets[l]);

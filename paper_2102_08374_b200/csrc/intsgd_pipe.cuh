@@ -49,6 +49,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+// Programmatic dependent launch: blocks until the grids this launch depends on have completed and their
+// writes are visible; returns at once for an ordinary launch.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 // Global -> shared bulk copy, completion signalled on an mbarrier of this CTA (no multicast).
 __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -200,7 +203,6 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
 
     const VecParams& P = PP.v;
     DevState* st = P.st;
-    if (st->status != INTSGD_OK) return;
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(&full_bar[s], 1);
@@ -211,6 +213,10 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
     }
     for (int i = threadIdx.x; i < INTSGD_MAX_WORKERS; i += blockDim.x) s_tab[i] = PP.tab.e[i];
     counters_init(s_cnt);   // includes a __syncthreads()
+    // Everything above needs only the kernel's arguments.  When the launch was allowed to start before
+    // the step's scale kernel has finished, wait here for that kernel's writes (a no-op otherwise).
+    grid_dependency_wait();
+    if (st->status != INTSGD_OK) return;
 
     const int n = P.n;
     const int64_t tiles = PP.tiles;
