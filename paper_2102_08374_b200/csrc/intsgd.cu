@@ -170,8 +170,23 @@ int launch_scale(intsgd_ctx* ctx, double eta, double dx2_override, cudaStream_t 
                                                ctx->cfg.n);
         return after_launch(ctx, "scale_blocks_kernel");
     }
-    scale_kernel<<<1, 32, 0, s>>>(ctx->d_state, std::sqrt(dd), 2.0 * dn, dn, eta, ctx->cfg.beta, ctx->cfg.eps,
-                                  dx2_override, ctx->cfg.n);
+    // The scale kernel may be scheduled while the kernel before it on the stream is still running (it waits
+    // for that kernel's completion before it touches the state): its launch latency leaves the step's path.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1, 1, 1);
+    cfg.blockDim = dim3(32, 1, 1);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, scale_kernel, ctx->d_state, std::sqrt(dd), 2.0 * dn, dn, eta, ctx->cfg.beta,
+                                             ctx->cfg.eps, dx2_override, (int32_t)ctx->cfg.n);
+    if (e != cudaSuccess) {
+        std::snprintf(ctx->err, 256, "launch of scale_kernel failed: %s", cudaGetErrorString(e));
+        return INTSGD_ERR_CUDA;
+    }
     return after_launch(ctx, "scale_kernel");
 }
 

@@ -16,6 +16,8 @@ __global__ void scale_kernel(DevState* st, double sqrt_d, double two_n, double n
     // a dependent launch (the step's vector kernel) may begin its set-up now; it waits for this grid's
     // completion before it reads the state
     asm volatile("griddepcontrol.launch_dependents;");
+    // this launch may itself have started before the kernel in front of it has finished: wait for its writes
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     const double dx2 = (dx2_override >= 0.0) ? dx2_override : st->dx2;
     const double a = __dmul_rn(beta, st->r);

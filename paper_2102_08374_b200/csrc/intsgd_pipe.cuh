@@ -203,6 +203,8 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
 
     const VecParams& P = PP.v;
     DevState* st = P.st;
+    // the next step's scale kernel may be scheduled from now on; it waits for this grid to complete
+    asm volatile("griddepcontrol.launch_dependents;");
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(&full_bar[s], 1);
