@@ -264,3 +264,31 @@ def test_step_host_over_several_windows_matches_the_oracle(grad_dtype, rounding)
             assert np.array_equal(hx.numpy().view(np.uint32), x_ref.view(np.uint32))
             assert rel_close(st["dx2"], ref["dx2"]) and st["max_abs_agg"] == ref["max_abs_agg"]
             assert st["clip_count"] == ref["clip_count"] and st["step"] == k + 2
+
+
+@pytest.mark.parametrize("blocks", [0, 3])
+def test_steps_enqueued_back_to_back_equal_steps_run_one_by_one(blocks):
+    """Without a host synchronisation between them the kernels of consecutive steps are chained by
+    programmatic dependent launches (each may start while the one before is still running and waits before
+    it reads the state); the results must be those of steps separated by synchronisations."""
+    n, d, seed, eta, K = 4, (1 << 20) + 3, 23, 0.1, 25
+    rng = np.random.default_rng(29)
+    grads = [to_dev(rng.normal(0, 1e-2, d).astype(np.float32)) for _ in range(n)]
+    x0 = rng.normal(0, 1, d).astype(np.float32)
+    out = []
+    for sync_every_step in (False, True):
+        with pkg.IntSGD(n, d, seed=seed) as lib:
+            if blocks:
+                lib.intsgd_set_blocks([0, d // 3, d // 2 + 1, d])
+            x = to_dev(x0.copy())
+            agg = torch.zeros(d, dtype=torch.int32, device=dev())
+            for k in range(K):
+                lib.intsgd_step(grads, x, agg, eta_k=eta, mode=pkg.MODE_EXACT if k == 0 else pkg.MODE_FUSED)
+                if sync_every_step:
+                    lib.intsgd_get_stats()
+            st = lib.intsgd_get_stats()
+            out.append((to_host(x), to_host(agg), st))
+    (xa, agga, sa), (xb, aggb, sb) = out
+    assert np.array_equal(xa.view(np.uint32), xb.view(np.uint32)) and np.array_equal(agga, aggb)
+    for key in ("r", "dx2", "alpha", "c", "step", "max_abs_agg", "clip_count"):
+        assert sa[key] == sb[key], key
