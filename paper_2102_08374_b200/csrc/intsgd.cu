@@ -404,7 +404,62 @@ void launch_diana_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStr
     else
         diana_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
+// Pipelined IntDIANA: 512 consumers, 2 units each, 2 worker slots (gradient tile + shift tile) per stage, 3 stages.
+template <int GRAD, int ROUND>
+cudaError_t launch_diana_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
+    constexpr int NC = 512, UPT = 2, G = 2, NS = 3;
+    auto kernel = diana_pipe_kernel<GRAD, ROUND, NC, UPT, G, NS>;
+    const int smem = NS * G * NC * UPT * (((GRAD == INTSGD_GRAD_F32) ? 16 : 8) + 16);
+    static bool configured[kMaxDevices] = {};
+    const int dev = ctx->cfg.device;
+    if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+    }
+    PP.tiles = (PP.units + NC * UPT - 1) / (NC * UPT);
+    const int64_t grid = PP.tiles < ctx->sm_count ? PP.tiles : ctx->sm_count;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(NC + 32, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->follows_scale ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, PP);
+}
+template <int GRAD>
+cudaError_t launch_diana_pipe_r(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
+    switch (ctx->cfg.rounding) {
+        case INTSGD_ROUND_NEAREST: return launch_diana_pipe_t<GRAD, INTSGD_ROUND_NEAREST>(ctx, PP, s);
+        case INTSGD_ROUND_RANDOM16: return launch_diana_pipe_t<GRAD, INTSGD_ROUND_RANDOM16>(ctx, PP, s);
+        case INTSGD_ROUND_RANDOM_COMPARE: return launch_diana_pipe_t<GRAD, INTSGD_ROUND_RANDOM_COMPARE>(ctx, PP, s);
+        default: return launch_diana_pipe_t<GRAD, INTSGD_ROUND_RANDOM>(ctx, PP, s);
+    }
+}
+int launch_diana_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
+    PipeParams PP;
+    PP.v = P;
+    PP.tab = ctx->tab;
+    const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
+    int64_t units = P.d >> 2;
+    if (bf16) units &= ~(int64_t)1;   // bulk copies move multiples of 16 bytes
+    PP.units = units;
+    PP.tiles = 0;
+    PP.fast_limit = ctx->Lf;   // not used: nothing is deferred in this kernel
+    const cudaError_t e = bf16 ? launch_diana_pipe_r<INTSGD_GRAD_BF16>(ctx, PP, s) : launch_diana_pipe_r<INTSGD_GRAD_F32>(ctx, PP, s);
+    if (e != cudaSuccess) {
+        std::snprintf(ctx->err, 256, "diana_pipe_kernel launch failed: %s", cudaGetErrorString(e));
+        return INTSGD_ERR_CUDA;
+    }
+    return after_launch(ctx, "diana_pipe_kernel");
+}
+
 int launch_diana(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
+    if (ctx->fused_path != 1 && pipe_eligible(ctx, aligned, P.d)) return launch_diana_pipe(ctx, P, s);
     const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
     if (!bf16 && aligned) launch_diana_r<INTSGD_GRAD_F32, true>(ctx, P, grid, s);
@@ -757,7 +812,10 @@ int intsgd_diana_step(intsgd_ctx* ctx, const void* const* grads, float* const* h
     P.agg = agg;
     ctx->last_stream = s;
     if ((rc = launch_scale(ctx, eta_k, -1.0, s)) != INTSGD_OK) return rc;
-    return launch_diana(ctx, P, al, s);
+    ctx->follows_scale = true;
+    rc = launch_diana(ctx, P, al, s);
+    ctx->follows_scale = false;
+    return rc;
 }
 
 int intsgd_heuristic_step(intsgd_ctx* ctx, const void* const* grads, float* x, int32_t* agg, double eta_k,

@@ -14,6 +14,7 @@
 
 #include "intsgd_blocks.cuh"
 #include "intsgd_device.cuh"
+#include "intsgd_kernels.cuh"
 
 namespace intsgd {
 
@@ -176,6 +177,20 @@ __device__ __forceinline__ uint4 split16(uint32_t a, uint32_t b) {
     return make_uint4(a & 0xFFFFu, a >> 16, b & 0xFFFFu, b >> 16);
 }
 
+// The four draws of one unit of one worker from the thread's folded Philox state.  With 16-bit draws and
+// PAIR_SHARED the block `pw` of the thread's pair was computed once and unit k takes its half.
+template <int ROUND, bool PAIR_SHARED>
+__device__ __forceinline__ uint4 unit_draws(const PhiloxThreadPart& t, const uint4& e, const uint4& pw, int k, bool h,
+                                            const PhiloxKeys& K) {
+    if (ROUND == INTSGD_ROUND_RANDOM || ROUND == INTSGD_ROUND_RANDOM_COMPARE) return philox_finish(t, e, K);
+    if (ROUND == INTSGD_ROUND_RANDOM16) {
+        if (PAIR_SHARED) return k == 0 ? split16(pw.x, pw.y) : split16(pw.z, pw.w);
+        const uint4 r = philox_finish(t, e, K);
+        return h ? split16(r.z, r.w) : split16(r.x, r.y);
+    }
+    return make_uint4(0, 0, 0, 0);
+}
+
 template <int GRAD>
 __device__ __forceinline__ float4 lds_unit(const unsigned char* tile, int c) {
     if (GRAD == INTSGD_GRAD_F32) return *reinterpret_cast<const float4*>(tile + 16 * c);
@@ -261,15 +276,6 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         const float alpha = st->alpha, cdec = st->c;
         const uint32_t step = st->step;
         const BlockParams& bp = P.bp;
-        auto unit_draws = [&](const PhiloxThreadPart& t, const uint4& e, const uint4& pw, int k, bool h) -> uint4 {
-            if (ROUND == INTSGD_ROUND_RANDOM || ROUND == INTSGD_ROUND_RANDOM_COMPARE) return philox_finish(t, e, P.keys);
-            if (ROUND == INTSGD_ROUND_RANDOM16) {
-                if (kPairShared) return k == 0 ? split16(pw.x, pw.y) : split16(pw.z, pw.w);
-                const uint4 r = philox_finish(t, e, P.keys);
-                return h ? split16(r.z, r.w) : split16(r.x, r.y);
-            }
-            return make_uint4(0, 0, 0, 0);
-        };
         uint32_t s = 0, phase = 0;
         float max_sum = 0.0f;                                            // max |S| over fast-path units
         const bool count_overflow = P.agg_limit != 0x7FFFFFFF;          // int8 wire: count |S| > 127
@@ -350,7 +356,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
 #pragma unroll
                         for (int k = 0; k < UPT; ++k) {
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
-                            consume_unit<ROUND>(gv, a01[k], a23[k], unit_draws(tp[k], e, pw, k, half[k]), ua[k]);
+                            consume_unit<ROUND>(gv, a01[k], a23[k], unit_draws<ROUND, kPairShared>(tp[k], e, pw, k, half[k], P.keys), ua[k]);
                         }
                     }
                 } else {
@@ -362,7 +368,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                         for (int k = 0; k < UPT; ++k) {
                             if (!active[k]) continue;
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
-                            consume_unit<ROUND>(gv, a01[k], a23[k], unit_draws(tp[k], e, pw, k, half[k]), ua[k]);
+                            consume_unit<ROUND>(gv, a01[k], a23[k], unit_draws<ROUND, kPairShared>(tp[k], e, pw, k, half[k], P.keys), ua[k]);
                         }
                     }
                 }

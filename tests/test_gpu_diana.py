@@ -14,10 +14,11 @@ pytestmark = pytest.mark.gpu
 
 class DianaLockStep:
     def __init__(self, n, d, x0, *, grad_dtype=pkg.GRAD_F32, payload_dtype=pkg.PAYLOAD_I32,
-                 rounding=pkg.ROUND_RANDOM, beta=0.0, eps=0.0, seed=0, unaligned=False):
+                 rounding=pkg.ROUND_RANDOM, beta=0.0, eps=0.0, seed=0, unaligned=False, fused_path=0):
         self.n, self.d, self.unaligned = n, d, unaligned
         self.lib = pkg.IntSGD(n, d, grad_dtype=grad_dtype, payload_dtype=payload_dtype, rounding=rounding,
                               beta=beta, eps=eps, seed=seed)
+        self.lib.intsgd_set_fused_path(fused_path)     # 0: pipelined kernel when the pointers allow it; 1: direct kernel
         self.orc = oracle.OracleIntDIANA(n, d, beta=beta, eps=eps, seed=seed, payload_dtype=payload_dtype,
                                          rounding=rounding)
         self.x_ref = x0.copy()
@@ -57,11 +58,11 @@ class DianaLockStep:
         return st, ref
 
 
-@pytest.mark.parametrize("unaligned", [False, True])
+@pytest.mark.parametrize("unaligned,fused_path", [(False, 0), (False, 1), (True, 0)])
 @pytest.mark.parametrize("grad_dtype,payload_dtype,rounding", [
     (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM), (pkg.GRAD_BF16, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM),
     (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_NEAREST), (pkg.GRAD_BF16, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM16), (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM_COMPARE)])
-def test_diana_lockstep_on_heterogeneous_quadratics(unaligned, grad_dtype, payload_dtype, rounding):
+def test_diana_lockstep_on_heterogeneous_quadratics(unaligned, fused_path, grad_dtype, payload_dtype, rounding):
     """f_i(x) = |x - b_i|^2 / 2 with different b_i (heterogeneous data), full local gradients computed
     by the harness from the library's own iterate; several tiles and a ragged tail."""
     rng = np.random.default_rng(12)
@@ -73,7 +74,7 @@ def test_diana_lockstep_on_heterogeneous_quadratics(unaligned, grad_dtype, paylo
         return [synth.to_bf16_bits(g) for g in out] if grad_dtype == pkg.GRAD_BF16 else out
 
     ls = DianaLockStep(n, d, np.zeros(d, dtype=np.float32), grad_dtype=grad_dtype, payload_dtype=payload_dtype,
-                       rounding=rounding, seed=31, unaligned=unaligned)
+                       rounding=rounding, seed=31, unaligned=unaligned, fused_path=fused_path)
     try:
         ls.exact(grads(ls.x_ref), eta)
         biggest = []
@@ -86,10 +87,12 @@ def test_diana_lockstep_on_heterogeneous_quadratics(unaligned, grad_dtype, paylo
         ls.close()
 
 
-def test_diana_with_values_that_clip_and_non_finite_gradients():
+@pytest.mark.parametrize("fused_path", [0, 1])
+def test_diana_with_values_that_clip_and_non_finite_gradients(fused_path):
     rng = np.random.default_rng(13)
     n, d, eta = 3, 40_003, 0.1
-    ls = DianaLockStep(n, d, rng.normal(0, 1, d).astype(np.float32), payload_dtype=pkg.PAYLOAD_I8, beta=0.9, eps=1e-8, seed=5)
+    ls = DianaLockStep(n, d, rng.normal(0, 1, d).astype(np.float32), payload_dtype=pkg.PAYLOAD_I8, beta=0.9, eps=1e-8, seed=5,
+                       fused_path=fused_path)
     try:
         ls.exact([rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)], eta)
         seen_clip = seen_nonf = 0
