@@ -33,8 +33,8 @@ HBM_FALLBACK_GBS = 6650.0
 # command and figures in profiles/fused_pipe_kernel_d24_n16_ncu_full.md): bytes per coordinate of the
 # captured case (d = 2^24, n = 16, fp32, int32 aggregate), valid for the kernel sources with this hash.
 # Any change to the kernel sources makes `roofline.traffic` null until the counters are taken again.
-NCU_TRAFFIC = {"sources_sha256": "89ae7eff1f9a109b067b14ffa26f3e1847d8a5b8e41127d99d9d9ac78462f68a",
-               "bytes_per_coordinate": 1.265289e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
+NCU_TRAFFIC = {"sources_sha256": "e876b48a8d7bd734868d0d17ee223a2e2c909f07d4f1e8d621b2454acc7dd95f",
+               "bytes_per_coordinate": 1.264733e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
 
 
 def kernel_sources_hash():
@@ -296,6 +296,11 @@ def main():
                 "algorithmic_bytes_per_launch": bytes_per_launch, "kernel_ms_avg": avg_ms,
                 "kernel_ms_median": statistics.median(per_step_ms),
                 "note": "per-step CUDA-event time (one-thread scale kernel + the vector kernel(s))"}
+    if clocks and clocks.get("sm_mhz"):
+        # The random-rounding kernel is co-limited by instruction issue (Philox): its time follows the SM clock.
+        # SM clocks spent per worker unit (4 gradient elements of one worker), from the clock sampled under load.
+        sms = torch.cuda.get_device_properties(device).multi_processor_count
+        roofline["sm_clocks_per_worker_unit"] = avg_ms * 1e-3 * clocks["sm_mhz"] * 1e6 * sms / (n * d / 4)
 
     # ---- the other rounding modes on the same buffers, short bursts (context for the headline; 1 GPU only) ----
     variants = None
