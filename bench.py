@@ -14,6 +14,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -175,23 +176,42 @@ def oracle_sample_throughput(n, d, sample_log2, grad_dtype, payload, rounding, s
 
 
 def run_reference(args):
-    """The reference arm: the CPU oracle, single-threaded, on a bounded sample per step."""
+    """The reference arm: the CPU oracle as it stands, single-threaded, W untimed and exactly K timed steps,
+    each over a window of the workload sized so that the whole run takes about a minute or two."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    import numpy as np
+    import oracle
+    from paper_2102_08374_b200 import synth
     n, d = args.workers, 1 << args.log2d
-    sample_log2 = min(args.cpu_sample_log2, 22)
-    for _ in range(max(args.warmup, 0) and 1):
-        oracle_sample_throughput(n, d, 16, args.grad, args.payload, args.rounding)
-    times, elems = [], 0
-    for _ in range(max(1, min(args.steps, 8))):
-        v, dt, desc = oracle_sample_throughput(n, d, sample_log2, args.grad, args.payload, args.rounding)
-        times.append(dt)
-        elems = n * min(d, 1 << sample_log2)
-    value = elems * len(times) / sum(times)
+    K, W = max(args.steps, 1), max(args.warmup, 0)
+    # about 1e9 gradient elements in all (the oracle does 1-2e7 per second and core), a power of two per step
+    per_step = 1.0e9 / ((K + W) * n)
+    sample_log2 = max(10, min(22, args.log2d, int(math.floor(math.log2(max(per_step, 1.0))))))
+    w = 1 << sample_log2
+    grads = [synth.bucket_gradient(i, w) for i in range(n)]
+    if args.grad == "bf16":
+        grads = [synth.to_bf16_bits(g) for g in grads]
+    x = synth.iterate(w)
+    pd = oracle.PAYLOAD_I8 if args.payload == "int8" else oracle.PAYLOAD_I32
+    rd = {"nearest": oracle.ROUND_NEAREST, "random16": oracle.ROUND_RANDOM16,
+          "compare": oracle.ROUND_RANDOM_COMPARE}.get(args.rounding, oracle.ROUND_RANDOM)
+
+    def one_step(k):
+        oracle.step_window(grads, x, np.float32(700.0), np.float32(1e-5), step=k, seed=77, payload_dtype=pd, rounding=rd)
+
+    for k in range(W):
+        one_step(1 + k)
+    t0 = time.perf_counter()
+    for k in range(K):
+        one_step(1 + W + k)
+    seconds = time.perf_counter() - t0
+    value = n * w * K / seconds
+    desc = f"each step covers the first 2^{sample_log2} coordinates of all {n} workers ({n * w} elements)"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": len(times), "warmup": 1, "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True,
+        "steps": K, "warmup": W, "ms_per_step": 1e3 * seconds / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": workload_config(args),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
