@@ -51,7 +51,7 @@ def traffic_per_launch(args, d):
     """Measured DRAM bytes per launch, scaled to d (traffic is proportional to d), or None."""
     t = NCU_TRAFFIC
     same = (args.workers == t["workers"] and args.grad == t["grad"] and args.mode == t["mode"]
-            and args.rounding == "random")
+            and args.rounding == "random" and args.kind == "intsgd")
     if not same or kernel_sources_hash() != t["sources_sha256"]:
         return None
     return t["bytes_per_coordinate"] * d
@@ -68,6 +68,11 @@ def parse_args():
     p.add_argument("--payload", default="int32", choices=["int32", "int8"])
     p.add_argument("--grad", default="f32", choices=["f32", "bf16"])
     p.add_argument("--mode", default="fused", choices=["fused", "two_kernel"])
+    p.add_argument("--kind", default="intsgd", choices=["intsgd", "diana", "heuristic", "blocks"],
+                   help="which step is timed: Algorithm 1 (default, the headline), the IntDIANA step (Algorithm 3), "
+                        "the heuristic SwitchML-style step (profiling pass + fused pass) or block-wise scales (Algorithm 2)")
+    p.add_argument("--num-bits", type=int, default=16, help="--kind heuristic: bits of the heuristic rule")
+    p.add_argument("--num-blocks", type=int, default=62, help="--kind blocks: equal contiguous blocks")
     p.add_argument("--rounding", default="random", choices=["random", "nearest", "random16", "compare"],
                    help="random16 = the optional 16-bit draw stream; compare = Int(t) drawn by comparing a 24-bit "
                         "uniform with the fractional part (both: a different random stream; not the default)")
@@ -144,12 +149,17 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def algorithmic_bytes_per_coordinate(n, grad_bytes, payload_bytes, mode):
+def algorithmic_bytes_per_coordinate(n, grad_bytes, payload_bytes, mode, kind="intsgd"):
     """Bytes that must cross HBM per coordinate: n gradient reads, x read + write, aggregate write
-    (fused); plus n payload writes and n payload reads on the two-kernel path."""
+    (fused); plus n payload writes and n payload reads on the two-kernel path.  IntDIANA also reads and
+    writes the n local shifts and the global shift; the heuristic step reads every gradient twice."""
     base = n * grad_bytes + 12
     if mode == "two_kernel":
         base += 2 * n * payload_bytes
+    if kind == "diana":
+        base += 8 * n + 8
+    if kind == "heuristic":
+        base += n * grad_bytes
     return base
 
 
@@ -222,8 +232,10 @@ def run_reference(args):
 
 
 def workload_config(args):
+    kind = {"intsgd": "", "diana": ", IntDIANA step", "heuristic": f", heuristic scale with {args.num_bits} bits",
+            "blocks": f", block-wise scales over {args.num_blocks} blocks"}[args.kind]
     return {"workload": f"large-model bucket: d=2^{args.log2d} {args.grad} N(0,1e-3^2), n={args.workers} workers, "
-                        f"{args.payload} wire, {args.mode} path, {args.rounding} rounding",
+                        f"{args.payload} wire, {args.mode} path, {args.rounding} rounding{kind}",
             "d": 1 << args.log2d, "n_workers": args.workers, "grad_dtype": args.grad, "payload": args.payload,
             "mode": args.mode, "rounding": args.rounding,
             "l2": "inputs larger than L2 (gradients alone are n*d*4 bytes); no flush between iterations"}
@@ -271,9 +283,24 @@ def main():
     lib.intsgd_set_launch(args.threads, args.blocks_per_sm)
     stream = torch.cuda.current_stream().cuda_stream
 
+    h_local = h_global = None
+    if args.kind == "diana":
+        h_local = [torch.zeros(d, dtype=torch.float32, device=device) for _ in range(n)]
+        h_global = torch.zeros(d, dtype=torch.float32, device=device)
+    if args.kind == "blocks":
+        B = max(1, min(args.num_blocks, d))
+        lib.intsgd_set_blocks([(d * b) // B for b in range(B)] + [d])
+    if args.kind != "intsgd" and mode != pkg.MODE_FUSED:
+        raise SystemExit("--kind diana / heuristic / blocks run the fused path only")
+
     def step(k):
-        lib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=pkg.MODE_EXACT if k == 0 else mode,
-                        payload_scratch=scratch, stream=stream)
+        if k > 0 and args.kind == "diana":
+            lib.intsgd_diana_step(grads, h_local, h_global, x, agg, eta_k=args.eta, stream=stream)
+        elif k > 0 and args.kind == "heuristic":
+            lib.intsgd_heuristic_step(grads, x, agg, eta_k=args.eta, num_bits=args.num_bits, stream=stream)
+        else:
+            lib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=pkg.MODE_EXACT if k == 0 else mode,
+                            payload_scratch=scratch, stream=stream)
 
     def barrier():
         if dist is not None:
@@ -307,7 +334,7 @@ def main():
     st = lib.intsgd_get_stats()
     total_ms = replicas.max_over_ranks(dist, total_ms, device)
     value = world * n * d * K / (total_ms * 1e-3)
-    bytes_per_launch = algorithmic_bytes_per_coordinate(n, gb, pb, args.mode) * d
+    bytes_per_launch = algorithmic_bytes_per_coordinate(n, gb, pb, args.mode, args.kind) * d
     avg_ms = statistics.mean(per_step_ms)
     peak, peak_kind = measured_hbm_peak()
     achieved = bytes_per_launch / (avg_ms * 1e-3) / 1e9
@@ -324,7 +351,7 @@ def main():
 
     # ---- the other rounding modes on the same buffers, short bursts (context for the headline; 1 GPU only) ----
     variants = None
-    if world == 1 and not args.no_variants and mode == pkg.MODE_FUSED:
+    if world == 1 and not args.no_variants and mode == pkg.MODE_FUSED and args.kind == "intsgd":
         variants = []
         names = {"random": pkg.ROUND_RANDOM, "compare": pkg.ROUND_RANDOM_COMPARE, "random16": pkg.ROUND_RANDOM16,
                  "nearest": pkg.ROUND_NEAREST}
@@ -347,7 +374,7 @@ def main():
 
     # ---- end to end through the host-buffer entry point (rank-local; max over ranks) ----
     e2e = None
-    if not args.no_e2e and mode == pkg.MODE_FUSED:
+    if not args.no_e2e and mode == pkg.MODE_FUSED and args.kind == "intsgd":
         hg = [torch.empty(d, dtype=g.dtype, pin_memory=True) for g in grads]
         for h, g in zip(hg, grads):
             h.copy_(g)
@@ -371,7 +398,7 @@ def main():
         del hg, hx, hagg
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.kind == "intsgd":
         v, dt, desc = oracle_sample_throughput(n, d, args.cpu_sample_log2, args.grad, args.payload, args.rounding)
         cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": dt}
 
