@@ -34,8 +34,8 @@ HBM_FALLBACK_GBS = 6650.0
 # command and figures in profiles/fused_pipe_kernel_d24_n16_ncu_full.md): bytes per coordinate of the
 # captured case (d = 2^24, n = 16, fp32, int32 aggregate), valid for the kernel sources with this hash.
 # Any change to the kernel sources makes `roofline.traffic` null until the counters are taken again.
-NCU_TRAFFIC = {"sources_sha256": "e876b48a8d7bd734868d0d17ee223a2e2c909f07d4f1e8d621b2454acc7dd95f",
-               "bytes_per_coordinate": 1.264733e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
+NCU_TRAFFIC = {"sources_sha256": "814cfb67602a3a7f3fbd42e8e07cfa2ef11b35b2e45f9a2587e92c90d0795469",
+               "bytes_per_coordinate": 1.266082e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
 
 
 def kernel_sources_hash():

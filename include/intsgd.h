@@ -226,6 +226,14 @@ int intsgd_set_launch(intsgd_ctx* ctx, int32_t threads_per_block, int32_t blocks
  * by summation order. */
 int intsgd_set_fused_path(intsgd_ctx* ctx, int32_t path);
 
+/* Diagnostic of the failure path.  Every wait inside the pipelined kernels is bounded; when one gives up the
+ * kernel sets a sticky flag, lets its copies in flight land and returns, and intsgd_get_stats reports
+ * INTSGD_ERR_TIMEOUT until intsgd_set_state clears the flag.  This call enqueues a one-thread kernel that runs
+ * the same bounded wait (64 polls) on a barrier that nothing ever completes, so that a caller can check, without
+ * any fault on the GPU, that an expired wait surfaces as INTSGD_ERR_TIMEOUT and that the context stays usable.
+ * It touches no vector and no other state. */
+int intsgd_selftest_wait_expiry(intsgd_ctx* ctx, void* stream);
+
 /* Number of kernels this library has launched on the context since creation. */
 int64_t intsgd_launch_count(const intsgd_ctx* ctx);
 

@@ -981,6 +981,15 @@ int intsgd_get_stats(intsgd_ctx* ctx, intsgd_stats* out) {
     return INTSGD_OK;
 }
 
+int intsgd_selftest_wait_expiry(intsgd_ctx* ctx, void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    ctx->last_stream = s;
+    wait_expiry_kernel<<<1, 32, 0, s>>>(ctx->d_state, 64u);
+    return after_launch(ctx, "wait_expiry_kernel");
+}
+
 int intsgd_get_state(intsgd_ctx* ctx, intsgd_state* out) {
     if (!ctx || !out) return INTSGD_ERR_INVALID_ARG;
     intsgd_stats s;

@@ -509,4 +509,16 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
     else grid_finalize(acc, st, P.partials, true, P.window_flags);
 }
 
+// Diagnostic: the bounded wait on a barrier that nothing completes.  One thread polls `polls` times, then
+// reports the expiry exactly as the step kernels do (sticky fault flag in the state) and returns.
+__global__ void wait_expiry_kernel(DevState* st, uint32_t polls) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x != 0) return;
+    mbar_init(&bar, 1);
+    mbar_fence_init();
+    bool done = false;
+    for (uint32_t i = 0; i < polls && !done; ++i) done = mbar_try_wait(&bar, 0u);   // mbar_wait with a short limit
+    if (!done) atomicExch(&st->fault, 1);
+}
+
 }  // namespace intsgd

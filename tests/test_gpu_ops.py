@@ -188,3 +188,33 @@ def test_misaligned_to_element_size_is_an_error_not_a_fault():
         with pytest.raises(pkg.IntSGDError):
             lib.intsgd_step([buf], x, None, eta_k=0.1, mode=pkg.MODE_TWO_KERNEL)   # no scratch
         assert "scratch" in lib.intsgd_last_error()
+
+
+def test_an_expired_wait_is_reported_and_the_context_stays_usable():
+    """The failure path without a GPU fault: the library's bounded wait runs out on a barrier that nothing
+    completes; the status is INTSGD_ERR_TIMEOUT until the state is set again, and the context then steps
+    exactly like a fresh one."""
+    n, d, eta, seed = 3, 5000, 0.1, 11
+    rng = np.random.default_rng(21)
+    grads = [to_dev(rng.normal(0, 1e-2, d).astype(np.float32)) for _ in range(n)]
+    x0 = rng.normal(0, 1, d).astype(np.float32)
+
+    def two_steps(lib):
+        x, agg = to_dev(x0.copy()), torch.zeros(d, dtype=torch.int32, device=dev())
+        lib.intsgd_step(grads, x, None, eta_k=eta, mode=pkg.MODE_EXACT)
+        lib.intsgd_step(grads, x, agg, eta_k=eta)
+        return to_host(x), to_host(agg), lib.intsgd_get_stats()
+
+    with pkg.IntSGD(n, d, seed=seed) as lib:
+        lib.intsgd_selftest_wait_expiry()
+        for _ in range(2):   # sticky
+            with pytest.raises(pkg.IntSGDError) as err:
+                lib.intsgd_get_stats()
+            assert err.value.code == pkg.ERR_TIMEOUT
+        lib.intsgd_set_state(r=0.0, dx2=0.0, alpha=0.0, c=0.0, step=0)
+        assert lib.intsgd_get_stats()["step"] == 0
+        x_a, agg_a, st_a = two_steps(lib)
+    with pkg.IntSGD(n, d, seed=seed) as fresh:
+        x_b, agg_b, st_b = two_steps(fresh)
+    assert np.array_equal(x_a.view(np.uint32), x_b.view(np.uint32)) and np.array_equal(agg_a, agg_b)
+    assert st_a["alpha"] == st_b["alpha"] and st_a["dx2"] == st_b["dx2"] and st_a["step"] == st_b["step"] == 2
