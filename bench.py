@@ -35,7 +35,9 @@ HBM_FALLBACK_GBS = 6650.0
 # captured case (d = 2^24, n = 16, fp32, int32 aggregate), valid for the kernel sources with this hash.
 # Any change to the kernel sources makes `roofline.traffic` null until the counters are taken again.
 NCU_TRAFFIC = {"sources_sha256": "814cfb67602a3a7f3fbd42e8e07cfa2ef11b35b2e45f9a2587e92c90d0795469",
-               "bytes_per_coordinate": 1.266082e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused"}
+               "bytes_per_coordinate": 1.266082e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused",
+               # smsp__inst_executed.sum of the same capture: warp instructions per launch -> thread instructions per element
+               "instructions_per_element": 136.115e6 * 32 / (16 * (1 << 24))}
 
 
 def kernel_sources_hash():
@@ -348,6 +350,15 @@ def main():
         # SM clocks spent per worker unit (4 gradient elements of one worker), from the clock sampled under load.
         sms = torch.cuda.get_device_properties(device).multi_processor_count
         roofline["sm_clocks_per_worker_unit"] = avg_ms * 1e-3 * clocks["sm_mhz"] * 1e6 * sms / (n * d / 4)
+        if roofline["traffic"] is not None:
+            # second limit: instruction issue (4 schedulers x 32 lanes per SM and clock, at the clock sampled under load)
+            ipe = NCU_TRAFFIC["instructions_per_element"]
+            issued = ipe * n * d / (avg_ms * 1e-3)
+            peak_issue = sms * 128 * clocks["sm_mhz"] * 1e6
+            roofline["co_limit"] = {"bound": "alu", "achieved": issued / 1e12, "peak": peak_issue / 1e12,
+                                    "unit": "T thread-instructions/s", "frac": issued / peak_issue,
+                                    "instructions_per_element": ipe,
+                                    "note": "instruction count from the ncu capture; peak = SMs x 128 lanes x sampled SM clock"}
 
     # ---- the other rounding modes on the same buffers, short bursts (context for the headline; 1 GPU only) ----
     variants = None
