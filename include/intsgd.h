@@ -49,7 +49,7 @@ extern "C" {
 #define INTSGD_ERR_ALIGN            -2   /* pointer not aligned to its element size */
 #define INTSGD_ERR_CUDA             -3   /* a CUDA runtime call failed; see intsgd_last_error */
 #define INTSGD_ERR_SCALE_NONFINITE  -4   /* alpha_k or c_k not finite or not positive; step not applied */
-#define INTSGD_ERR_UNSUPPORTED      -5   /* valid request this build does not implement */
+#define INTSGD_ERR_UNSUPPORTED      -5   /* valid request that is not implemented */
 #define INTSGD_ERR_TOO_LARGE        -7   /* intsgd_sqdiff_noalloc: d exceeds INTSGD_NOALLOC_MAX_D */
 #define INTSGD_ERR_TIMEOUT          -6   /* a bounded wait inside a kernel gave up; that step's results are
                                             invalid; sticky until intsgd_set_state */
