@@ -83,6 +83,7 @@ def parse_args():
     p.add_argument("--cpu-sample-log2", type=int, default=24,
                    help="coordinates of the oracle sample (all workers), as a power of two")
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-cpu-all-cores", action="store_true", help="skip the all-cores leg of the CPU baseline")
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--no-variants", action="store_true", help="skip the short runs of the other rounding modes")
     p.add_argument("--threads", type=int, default=0)
@@ -185,6 +186,49 @@ def oracle_sample_throughput(n, d, sample_log2, grad_dtype, payload, rounding, s
     oracle.step_window(grads, x, np.float32(700.0), np.float32(1e-5), step=1, seed=seed, payload_dtype=pd, rounding=rd)
     dt = time.perf_counter() - t
     return n * w / dt, dt, f"one step on the first 2^{sample_log2} coordinates of all {n} workers ({n * w} elements)"
+
+
+def _oracle_window_task(task):
+    """Runs in a spawned worker process: the unchanged oracle on one coordinate window of the sample.
+    Returns the wall-clock interval of the timed call (inputs are drawn before it starts)."""
+    import numpy as np
+    import oracle
+    from paper_2102_08374_b200 import synth
+    n, j0, count, grad_dtype, payload, rounding, seed = task
+    grads = [synth.bucket_gradient(i, count, seed_base=7000 + 64 * (j0 // max(count, 1))) for i in range(n)]
+    if grad_dtype == "bf16":
+        grads = [synth.to_bf16_bits(g) for g in grads]
+    x = synth.iterate(count, seed=8000 + j0 // max(count, 1))
+    pd = oracle.PAYLOAD_I8 if payload == "int8" else oracle.PAYLOAD_I32
+    rd = {"nearest": oracle.ROUND_NEAREST, "random16": oracle.ROUND_RANDOM16,
+          "compare": oracle.ROUND_RANDOM_COMPARE}.get(rounding, oracle.ROUND_RANDOM)
+    oracle.step_window([g[:256] for g in grads], x[:256].copy(), np.float32(700.0), np.float32(1e-5), step=1,
+                       seed=seed, j0=j0, payload_dtype=pd, rounding=rd)    # load the library, touch the code
+    t0 = time.time()
+    oracle.step_window(grads, x, np.float32(700.0), np.float32(1e-5), step=1, seed=seed, j0=j0, payload_dtype=pd,
+                       rounding=rd)
+    return t0, time.time()
+
+
+def oracle_all_cores_throughput(n, d, sample_log2, grad_dtype, payload, rounding, seed=77):
+    """The same oracle on all host cores: the sample's coordinates are cut into one window per core, and
+    each window is stepped by an unchanged single-threaded oracle in its own (spawned) process -- valid
+    because the random stream is addressed by (seed, step, worker, coordinate).  Returns
+    (elements/s, cores, description); the time runs from the first window's start to the last one's end."""
+    import multiprocessing as mp
+    cores = max(1, min(os.cpu_count() or 1, 64))
+    w = min(d, 1 << sample_log2)
+    count = max(w // cores // 4 * 4, 4)
+    tasks = [(n, k * count, count, grad_dtype, payload, rounding, seed) for k in range(cores)]
+    pool = mp.get_context("spawn").Pool(cores)
+    try:
+        spans = pool.map_async(_oracle_window_task, tasks, chunksize=1).get(timeout=180)
+    finally:
+        pool.terminate()
+        pool.join()
+    seconds = max(t1 for _, t1 in spans) - min(t0 for t0, _ in spans)
+    return n * count * cores / seconds, cores, (f"{cores} windows of {count} coordinates x {n} workers, one process "
+                                                f"per core ({n * count * cores} elements, {seconds:.2f} s)")
 
 
 def run_reference(args):
@@ -412,6 +456,12 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline and args.kind == "intsgd":
         v, dt, desc = oracle_sample_throughput(n, d, args.cpu_sample_log2, args.grad, args.payload, args.rounding)
         cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": dt}
+        if not args.no_cpu_all_cores:
+            try:
+                va, cores, desca = oracle_all_cores_throughput(n, d, args.cpu_sample_log2, args.grad, args.payload, args.rounding)
+                cpu["all_cores"] = {"value": va, "unit": UNIT, "cores": cores, "sample": desca}
+            except Exception as exc:   # a box that cannot spawn processes still reports the one-thread figure
+                cpu["all_cores"] = {"unavailable": repr(exc)}
 
     if rank == 0:
         line = {
