@@ -377,7 +377,10 @@ def main():
     clocks = sampler.stop(t_wall0, t_wall1)
     total_ms = events[0].elapsed_time(events[K])
     per_step_ms = [events[k].elapsed_time(events[k + 1]) for k in range(K)]
-    st = lib.intsgd_get_stats()
+    st = lib.intsgd_get_stats()   # raises if a step was refused (scale not finite) or a bounded wait expired
+    expected_steps = 1 + max(args.warmup, 3) + K
+    if st["step"] != expected_steps:
+        raise SystemExit(f"bench.py: {st['step']} steps were applied, {expected_steps} were enqueued: the timing is void")
     total_ms = replicas.max_over_ranks(dist, total_ms, device)
     value = world * n * d * K / (total_ms * 1e-3)
     bytes_per_launch = algorithmic_bytes_per_coordinate(n, gb, pb, args.mode, args.kind) * d
