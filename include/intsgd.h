@@ -50,9 +50,9 @@ extern "C" {
 #define INTSGD_ERR_CUDA             -3   /* a CUDA runtime call failed; see intsgd_last_error */
 #define INTSGD_ERR_SCALE_NONFINITE  -4   /* alpha_k or c_k not finite or not positive; step not applied */
 #define INTSGD_ERR_UNSUPPORTED      -5   /* valid request that is not implemented */
-#define INTSGD_ERR_TOO_LARGE        -7   /* intsgd_sqdiff_noalloc: d exceeds INTSGD_NOALLOC_MAX_D */
 #define INTSGD_ERR_TIMEOUT          -6   /* a bounded wait inside a kernel gave up; that step's results are
                                             invalid; sticky until intsgd_set_state */
+#define INTSGD_ERR_TOO_LARGE        -7   /* intsgd_sqdiff_noalloc: d exceeds INTSGD_NOALLOC_MAX_D */
 
 /* enums (plain ints in the structs) */
 #define INTSGD_GRAD_F32      0
@@ -248,10 +248,15 @@ int64_t intsgd_launch_count(const intsgd_ctx* ctx);
  *   out       : device, one double, 8-byte aligned; receives sum_j fl32(x_j - x_prev_j)^2 in fp64
  *   d         : 1 .. INTSGD_NOALLOC_MAX_D; larger -> INTSGD_ERR_TOO_LARGE, nothing is enqueued
  * Works on the current device and enqueues on `stream` without synchronising.  The first call on
- * each device looks up the array's device address (cudaGetSymbolAddress); make that first call
- * before any stream capture.  All calls on a device share the array: it keeps the previous call's
- * partial sums, its arrival counter is cleared on `stream` before every launch, and two calls that
- * overlap on the GPU race.  The summation order depends on d only. */
+ * each device looks up the array's device address (cudaGetSymbolAddress) and keeps it for the life of the
+ * process: it assumes that the device's primary context is not destroyed (cudaDeviceReset) while the
+ * library is in use.  The entry point has two kernels (both pointers 16-byte aligned / otherwise), and the
+ * CUDA runtime may load each on its first launch.  Make the first call on a device, and the first call of
+ * each alignment kind that will be used, before any stream capture.  All calls on a device share the
+ * array: it keeps the previous call's partial sums, its arrival counter is cleared on `stream` before
+ * every launch, and two calls that overlap on the GPU race.  The summation order depends only on d and on
+ * whether both x and x_prev are 16-byte aligned (the two kernels split a block's coordinates differently
+ * over its threads), never on the GPU or on scheduling. */
 #define INTSGD_NOALLOC_MAX_D ((int64_t)1 << 28)
 int intsgd_sqdiff_noalloc(const float* x, const float* x_prev, int64_t d, double* out, void* stream);
 

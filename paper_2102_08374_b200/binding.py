@@ -1,6 +1,9 @@
 """Thin ctypes binding of ``libintsgd.so`` (the C ABI declared in ``include/intsgd.h``).
 
-Argument marshalling only: every step of the IntSGD path runs in the CUDA kernels.  There is no
+Argument marshalling only: every step of the IntSGD path runs in the CUDA kernels.  Before an address
+crosses the C ABI the binding checks what the library cannot see from a bare pointer: the number of
+buffers in a list, element type, length, contiguity and which device a tensor lives on
+(``IntSGDError`` with ``ERR_INVALID_ARG``; nothing is launched).  There is no
 CPU fallback; if the library cannot be loaded, or no CUDA device is present when a context is
 created, an exception is raised.
 """
@@ -122,6 +125,56 @@ def _addr(t) -> int | None:
     raise TypeError(f"cannot take the address of {type(t)}")
 
 
+# Element types a buffer may have for each role.  bf16 gradients may also be handed over as their 16-bit
+# patterns (int16 / uint16 carriers).
+_DTYPES = {
+    "f32": ("float32",), "bf16": ("bfloat16", "int16", "uint16"), "i32": ("int32",), "i8": ("int8",),
+    "f64": ("float64",),
+}
+
+
+def _bad(msg: str):
+    raise IntSGDError(ERR_INVALID_ARG, msg)
+
+
+def _check_buffer(t, what: str, kind: str, count: int, device: int | None):
+    """Host-side argument check of one vector before its address crosses the C ABI.
+
+    ``device`` is the CUDA ordinal the buffer must live on, or None for a host buffer.  A raw integer
+    address cannot be inspected and is passed through (the library still checks NULL and alignment);
+    None is left to the library as well, which reports it as a NULL pointer.
+    """
+    if t is None or isinstance(t, int):
+        return
+    name = str(getattr(t, "dtype", "")).replace("torch.", "")
+    if name not in _DTYPES[kind]:
+        _bad(f"{what}: element type {name or type(t).__name__} where {' / '.join(_DTYPES[kind])} is expected")
+    numel = t.numel() if hasattr(t, "numel") else int(getattr(t, "size", 0))
+    if numel < count:
+        _bad(f"{what}: {numel} elements where at least {count} are needed")
+    if hasattr(t, "is_contiguous"):
+        if not t.is_contiguous():
+            _bad(f"{what}: not contiguous")
+    elif hasattr(t, "flags") and not t.flags["C_CONTIGUOUS"]:
+        _bad(f"{what}: not contiguous")
+    on_cuda = bool(getattr(t, "is_cuda", False))
+    if device is None:
+        if on_cuda:
+            _bad(f"{what}: a device tensor where a host buffer is expected")
+    else:
+        if not on_cuda:
+            _bad(f"{what}: a host buffer where a tensor on cuda:{device} is expected")
+        if t.device.index != device:
+            _bad(f"{what}: lives on cuda:{t.device.index}, the context is on cuda:{device}")
+
+
+def _check_list(seq, what: str, kind: str, count: int, device: int | None, n: int):
+    if seq is None or len(seq) != n:
+        _bad(f"{what}: {0 if seq is None else len(seq)} buffers where the context has n = {n} workers")
+    for i, t in enumerate(seq):
+        _check_buffer(t, f"{what}[{i}]", kind, count, device)
+
+
 def _ptr_array(seq):
     return (C.c_void_p * len(seq))(*[_addr(t) for t in seq])
 
@@ -134,6 +187,11 @@ def intsgd_sqdiff_noalloc(x, x_prev, d, out, stream=None) -> None:
     ``out``: one device double.  ``d`` may not exceed ``NOALLOC_MAX_D``.  Calls on one device share
     the scratch, so they must not overlap on the GPU.
     """
+    if isinstance(d, int) and 1 <= d <= NOALLOC_MAX_D:   # other sizes are refused by the library itself
+        where = next((t.device.index for t in (x, x_prev, out) if getattr(t, "is_cuda", False)), 0)
+        _check_buffer(x, "x", "f32", d, where)
+        _check_buffer(x_prev, "x_prev", "f32", d, where)
+        _check_buffer(out, "out", "f64", 1, where)
     rc = load().intsgd_sqdiff_noalloc(_addr(x), _addr(x_prev), d, _addr(out), stream)
     if rc != OK:
         what = {ERR_TOO_LARGE: f"d = {d} exceeds the fixed scratch (max {NOALLOC_MAX_D} coordinates)",
@@ -159,6 +217,9 @@ class IntSGD:
             raise IntSGDError(rc, msg)
         self.n, self.d = n, d
         self.num_blocks = 0
+        self._g = "bf16" if grad_dtype == GRAD_BF16 else "f32"
+        self._p = "i8" if payload_dtype == PAYLOAD_I8 else "i32"
+        self._dev = device
 
     # -- lifetime ---------------------------------------------------------------------------
     def close(self):
@@ -183,34 +244,57 @@ class IntSGD:
             raise IntSGDError(rc, self._lib.intsgd_last_error(self._ctx).decode())
         return rc
 
+    def _check_x_agg(self, x, agg):
+        _check_buffer(x, "x", "f32", self.d, self._dev)
+        _check_buffer(agg, "agg", "i32", self.d, self._dev)
+
     # -- the calls of the C ABI -----------------------------------------------------------------
     def intsgd_scale(self, eta_k, dx2_override=-1.0, stream=None):
         self._check(self._lib.intsgd_scale(self._ctx, eta_k, dx2_override, stream))
 
     def intsgd_sqdiff(self, x, x_prev, stream=None):
+        _check_buffer(x, "x", "f32", self.d, self._dev)
+        _check_buffer(x_prev, "x_prev", "f32", self.d, self._dev)
         self._check(self._lib.intsgd_sqdiff(self._ctx, _addr(x), _addr(x_prev), stream))
 
     def intsgd_encode(self, worker, grad, payload, alpha_override=math.nan, stream=None):
+        _check_buffer(grad, "grad", self._g, self.d, self._dev)
+        _check_buffer(payload, "payload", self._p, self.d, self._dev)
         self._check(self._lib.intsgd_encode(self._ctx, worker, _addr(grad), _addr(payload),
                                             alpha_override, stream))
 
     def intsgd_aggregate(self, payloads, x, agg=None, stream=None):
+        _check_list(payloads, "payloads", self._p, self.d, self._dev, self.n)
+        self._check_x_agg(x, agg)
         self._check(self._lib.intsgd_aggregate(self._ctx, _ptr_array(payloads), _addr(x), _addr(agg), stream))
 
     def intsgd_step(self, grads, x, agg=None, *, eta_k, mode=MODE_FUSED, payload_scratch=None, stream=None):
+        _check_list(grads, "grads", self._g, self.d, self._dev, self.n)
+        self._check_x_agg(x, agg)
+        if payload_scratch is not None:
+            _check_list(payload_scratch, "payload_scratch", self._p, self.d, self._dev, self.n)
         scratch = _ptr_array(payload_scratch) if payload_scratch is not None else None
         self._check(self._lib.intsgd_step(self._ctx, _ptr_array(grads), scratch, _addr(x), _addr(agg),
                                           eta_k, mode, stream))
 
     def intsgd_diana_step(self, grads, h_local, h_global, x, agg=None, *, eta_k, stream=None):
+        _check_list(grads, "grads", self._g, self.d, self._dev, self.n)
+        _check_list(h_local, "h_local", "f32", self.d, self._dev, self.n)
+        _check_buffer(h_global, "h_global", "f32", self.d, self._dev)
+        self._check_x_agg(x, agg)
         self._check(self._lib.intsgd_diana_step(self._ctx, _ptr_array(grads), _ptr_array(h_local), _addr(h_global),
                                                 _addr(x), _addr(agg), eta_k, stream))
 
     def intsgd_heuristic_step(self, grads, x, agg=None, *, eta_k, num_bits, stream=None):
+        _check_list(grads, "grads", self._g, self.d, self._dev, self.n)
+        self._check_x_agg(x, agg)
         self._check(self._lib.intsgd_heuristic_step(self._ctx, _ptr_array(grads), _addr(x), _addr(agg), eta_k,
                                                     num_bits, stream))
 
     def intsgd_step_host(self, host_grads, host_x, host_agg=None, *, eta_k, mode=MODE_FUSED, stream=None):
+        _check_list(host_grads, "host_grads", self._g, self.d, None, self.n)
+        _check_buffer(host_x, "host_x", "f32", self.d, None)
+        _check_buffer(host_agg, "host_agg", "i32", self.d, None)
         self._check(self._lib.intsgd_step_host(self._ctx, _ptr_array(host_grads), _addr(host_x),
                                                _addr(host_agg), eta_k, mode, stream))
 

@@ -1,5 +1,6 @@
 // Host side of the IntSGD step library: argument checks, launch shapes, the C ABI of intsgd.h.
 // Every step of the path runs in the kernels of intsgd_kernels.cuh; there is no CPU fallback.
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -262,12 +263,14 @@ cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s)
     auto kernel = fused_pipe_kernel<GRAD, ROUND, BLOCKS, S.nc, S.upt, S.g, S.ns>;
     const int unit_bytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
     const int smem = S.ns * S.g * S.nc * S.upt * unit_bytes;
-    static bool configured[kMaxDevices] = {};   // per instantiation and device: the opt-in to large shared memory
+    // per instantiation and device: the opt-in to large shared memory (contexts on other threads may race here:
+    // setting the attribute twice is harmless, the flag itself is atomic)
+    static std::atomic<bool> configured[kMaxDevices] = {};
     const int dev = ctx->cfg.device;
-    if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+    if (dev < 0 || dev >= kMaxDevices || !configured[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+        if (dev >= 0 && dev < kMaxDevices) configured[dev].store(true, std::memory_order_release);
     }
     PP.tiles = (PP.units + S.nc * S.upt - 1) / (S.nc * S.upt);
     int64_t grid = PP.tiles < ctx->sm_count ? PP.tiles : ctx->sm_count;
@@ -410,12 +413,12 @@ cudaError_t launch_diana_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStrea
     constexpr int NC = 512, UPT = 2, G = 2, NS = 3;
     auto kernel = diana_pipe_kernel<GRAD, ROUND, NC, UPT, G, NS>;
     const int smem = NS * G * NC * UPT * (((GRAD == INTSGD_GRAD_F32) ? 16 : 8) + 16);
-    static bool configured[kMaxDevices] = {};
+    static std::atomic<bool> configured[kMaxDevices] = {};
     const int dev = ctx->cfg.device;
-    if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+    if (dev < 0 || dev >= kMaxDevices || !configured[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+        if (dev >= 0 && dev < kMaxDevices) configured[dev].store(true, std::memory_order_release);
     }
     PP.tiles = (PP.units + NC * UPT - 1) / (NC * UPT);
     const int64_t grid = PP.tiles < ctx->sm_count ? PP.tiles : ctx->sm_count;
@@ -931,10 +934,17 @@ int intsgd_step_host(intsgd_ctx* ctx, const void* const* host_grads, float* host
     const size_t gbytes = d * grad_elem_size(ctx->cfg.grad_dtype);
     for (int i = 0; i < n; ++i)
         if (!host_grads[i]) return fail(ctx, INTSGD_ERR_INVALID_ARG, "host_grads[i] is NULL");
-    if (!ctx->stage_x) {
-        for (int i = 0; i < n; ++i) CUDA_TRY(ctx, cudaMalloc(&ctx->stage_grads[i], gbytes));
-        CUDA_TRY(ctx, cudaMalloc(&ctx->stage_x, d * sizeof(float)));
-        CUDA_TRY(ctx, cudaMalloc(&ctx->stage_agg, d * sizeof(int32_t)));
+    if (!ctx->stage_agg) {
+        // staging is all or nothing: a failed allocation releases what the attempt had obtained
+        cudaError_t e = cudaSuccess;
+        for (int i = 0; i < n && e == cudaSuccess; ++i)
+            if (!ctx->stage_grads[i]) e = cudaMalloc(&ctx->stage_grads[i], gbytes);
+        if (e == cudaSuccess && !ctx->stage_x) e = cudaMalloc((void**)&ctx->stage_x, d * sizeof(float));
+        if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->stage_agg, d * sizeof(int32_t));
+        if (e != cudaSuccess) {
+            free_staging(ctx);
+            return fail(ctx, INTSGD_ERR_CUDA, "intsgd_step_host: staging allocation failed: %s", cudaGetErrorString(e));
+        }
     }
     cudaStream_t s = (cudaStream_t)stream;
     if (d > (size_t)kHostWindow && ctx->bs.B == 0) {
@@ -994,8 +1004,8 @@ int intsgd_get_state(intsgd_ctx* ctx, intsgd_state* out) {
     if (!ctx || !out) return INTSGD_ERR_INVALID_ARG;
     intsgd_stats s;
     const int rc = intsgd_get_stats(ctx, &s);
-    if (rc != INTSGD_OK && rc != INTSGD_ERR_SCALE_NONFINITE) return rc;
-    *out = s.state;
+    // the state block has been read whenever get_stats got as far as its own status checks
+    if (rc == INTSGD_OK || rc == INTSGD_ERR_SCALE_NONFINITE || rc == INTSGD_ERR_TIMEOUT) *out = s.state;
     return rc;
 }
 

@@ -171,7 +171,7 @@ def test_unaligned_pointers_take_the_elementwise_path():
 def test_misaligned_to_element_size_is_an_error_not_a_fault():
     d = 64
     with pkg.IntSGD(1, d) as lib:
-        buf = torch.zeros(4 * d + 16, dtype=torch.uint8, device=dev())
+        buf = torch.zeros(d + 4, dtype=torch.float32, device=dev())
         x = torch.zeros(d, dtype=torch.float32, device=dev())
         with pytest.raises(pkg.IntSGDError) as e:
             lib.intsgd_step([buf.data_ptr() + 2], x, None, eta_k=0.1, mode=pkg.MODE_EXACT)
@@ -184,7 +184,7 @@ def test_misaligned_to_element_size_is_an_error_not_a_fault():
                 lib.intsgd_step([buf], x, None, eta_k=bad_eta, mode=pkg.MODE_FUSED)
             assert e.value.code == pkg.ERR_INVALID_ARG
         with pytest.raises(pkg.IntSGDError):
-            lib.intsgd_encode(1, buf, buf)          # worker out of range
+            lib.intsgd_encode(1, buf, torch.zeros(d, dtype=torch.int32, device=dev()))   # worker out of range
         with pytest.raises(pkg.IntSGDError):
             lib.intsgd_step([buf], x, None, eta_k=0.1, mode=pkg.MODE_TWO_KERNEL)   # no scratch
         assert "scratch" in lib.intsgd_last_error()

@@ -1,14 +1,16 @@
-"""intsgd_sqdiff_noalloc: the allocation-free norm entry point against intsgd_sqdiff.
+"""intsgd_sqdiff_noalloc: the allocation-free norm entry point against intsgd_sqdiff and against the CPU oracle.
 
 Collected last on purpose (file name): a failure here cannot hide a failure elsewhere.  The entry
 point exists for hosts that cannot call cudaMalloc and therefore cannot create a context; its
 scratch is a fixed array in the library that every call on the device shares, so the test calls it
-twice in a row on different data and expects both answers to match the context-based entry point.
+twice in a row on different data and expects both answers to match the context-based entry point, and
+the oracle's serial fp64 sum of the same vectors.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2102_08374_b200 as pkg
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +46,9 @@ def test_two_calls_in_a_row_match_the_context_entry_point():
     want = [_reference(x, x_prev) for x, x_prev in pairs]
     for g, w in zip(got, want):
         assert w > 0 and abs(g - w) <= REL * w, (g, w)
+    for g, (x, x_prev) in zip(got, pairs):   # and the oracle: serial fp64 sum of the squared fp32 differences
+        w = oracle.sqdiff(x.cpu().numpy(), x_prev.cpu().numpy())
+        assert abs(g - w) <= REL * w, (g, w)
     # an unaligned view (element-wise loads) and a repeat of the first case give the same answers
     x, x_prev = pairs[1]
     xb = torch.empty(x.numel() + 1, device=dev)[1:].copy_(x)
