@@ -6,8 +6,11 @@
 A step is one whole IntSGD iteration -- scale, encode, integer sum, decode, update, next-norm --
 over n workers' gradients of length d that are already in device memory (`value`), and the same
 step through the host-buffer entry point with the copies inside the timed region (`e2e`).
-Workload: the large-model bucket (d = 2^26 fp32 N(0, 1e-3^2), n = 16 workers, int32 aggregate,
-fused single-pass path).  With N > 1 (torchrun) every rank runs an independent replica on its own
+Workload: the largest row of the large-model bucket sweep (d = 2^28 fp32 N(0, 1e-3^2), n = 16 workers,
+16 GiB of gradients, int32 aggregate, fused single-pass path).  Two timings are printed: the K steps the
+command line asks for (a burst when K is small), and a segment of at least two seconds of back-to-back
+steps during which the board settles at its power cap (`roofline.sustained`), with the SM clock sampled
+through NVML across both.  With N > 1 (torchrun) every rank runs an independent replica on its own
 GPU: the path has no exchange step on one node, so there is no collective on the data path.
 """
 from __future__ import annotations
@@ -62,10 +65,10 @@ def traffic_per_launch(args, d):
 def parse_args():
     p = argparse.ArgumentParser()
     p.add_argument("--gpus", type=int, default=1)
-    p.add_argument("--steps", type=int, default=1000)
+    p.add_argument("--steps", type=int, default=50)
     p.add_argument("--warmup", type=int, default=5)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--log2d", type=int, default=26)
+    p.add_argument("--log2d", type=int, default=28)
     p.add_argument("--workers", type=int, default=16)
     p.add_argument("--payload", default="int32", choices=["int32", "int8"])
     p.add_argument("--grad", default="f32", choices=["f32", "bf16"])
@@ -80,6 +83,8 @@ def parse_args():
                         "uniform with the fractional part (both: a different random stream; not the default)")
     p.add_argument("--eta", type=float, default=0.1)
     p.add_argument("--e2e-steps", type=int, default=3)
+    p.add_argument("--sustain-seconds", type=float, default=2.0,
+                   help="length of the second timed segment (steps back to back, SM clock sampled); 0 = skip")
     p.add_argument("--cpu-sample-log2", type=int, default=24,
                    help="coordinates of the oracle sample (all workers), as a power of two")
     p.add_argument("--no-cpu-baseline", action="store_true")
@@ -103,53 +108,98 @@ def measured_hbm_peak():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and clock-event reasons while timed regions run: NVML from a thread (a few
+    milliseconds apart, so that a region of tens of milliseconds is covered), else nvidia-smi every 50 ms.
+    Reading only; no setting of the GPU is touched."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index, self.proc, self.lines = index, None, []
+    def __init__(self, index: int, uuid: str | None = None, period_s: float = 0.004):
+        self.index, self.uuid, self.period = index, uuid, period_s
+        self.samples = []      # (time, sm_mhz, max_mhz, watts, [reasons])
+        self.proc = self.thread = None
+        self.stop_flag = threading.Event()
+        self.source = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            h = None
+            if self.uuid:
+                for cand in (self.uuid, "GPU-" + self.uuid):
+                    try:
+                        h = pynvml.nvmlDeviceGetHandleByUUID(cand.encode() if isinstance(cand, str) else cand)
+                        break
+                    except Exception:
+                        h = None
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            mx = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            reasons_fn = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
+            float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))    # fails here if NVML cannot be read
+
+            def loop():
+                while not self.stop_flag.is_set():
+                    try:
+                        mhz = float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                        watts = pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0
+                        mask = int(reasons_fn(h))
+                        self.samples.append((time.time(), mhz, mx, watts, [n for b, n in self.REASONS.items() if mask & b]))
+                    except Exception:
+                        pass
+                    time.sleep(self.period)
+
+            self.thread = threading.Thread(target=loop, daemon=True)
+            self.thread.start()
+            self.source = "nvml"
+            return
+        except Exception:
+            self.thread = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
                  "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
+            self.source = "nvidia-smi"
         except Exception:
             self.proc = None
 
     def _pump(self):
-        for line in self.proc.stdout:
-            self.lines.append((time.time(), line.strip()))
-
-    def stop(self, t0=None, t1=None):
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for (t, line) in self.lines:
-            if t0 is not None and not (t0 - 0.05 <= t <= t1 + 0.1):
-                continue
-            parts = [s.strip() for s in line.split(",")]
-            if len(parts) < 7:
-                continue
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
             try:
-                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
-            except ValueError:
+                self.samples.append((time.time(), float(parts[0]), float(parts[1]), float(parts[2]),
+                                     [n for n, v in zip(names, parts[3:7]) if v.lower().startswith("active")]))
+            except (ValueError, IndexError):
                 continue
-            for name, v in zip(names, parts[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+    def stop(self):
+        self.stop_flag.set()
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        if self.thread:
+            self.thread.join(timeout=2)
+
+    def window(self, t0, t1):
+        """Summary of the samples taken between two wall-clock times."""
+        rows = [r for r in self.samples if t0 <= r[0] <= t1]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "power_w_max": None, "reasons": [], "samples": 0, "source": self.source}
+        reasons = sorted({n for r in rows for n in r[4]})
+        return {"sm_mhz": statistics.median(r[1] for r in rows), "sm_max_mhz": max(r[2] for r in rows),
+                "sm_mhz_min": min(r[1] for r in rows), "power_w_max": max(r[3] for r in rows), "reasons": reasons,
+                "samples": len(rows), "source": self.source}
 
 
 def algorithmic_bytes_per_coordinate(n, grad_bytes, payload_bytes, mode, kind="intsgd"):
@@ -164,6 +214,17 @@ def algorithmic_bytes_per_coordinate(n, grad_bytes, payload_bytes, mode, kind="i
     if kind == "heuristic":
         base += n * grad_bytes
     return base
+
+
+def wide_multiplies_per_worker_unit(args, n):
+    """32x32->64-bit multiplies of Philox4x32-10 per worker unit (4 gradient elements of one worker) on the path
+    `bench.py` times.  The pipelined kernels keep a thread on the same units for all workers: the unit's half of
+    rounds 1-2 (2 multiplies) is shared by the n workers, the worker's half comes from a table, rounds 3-10 cost
+    16.  With 16-bit draws one block serves two units.  Deterministic rounding draws nothing."""
+    if args.rounding == "nearest":
+        return 0.0
+    per = 16.0 + 2.0 / n
+    return per / 2 if args.rounding == "random16" else per
 
 
 # ------------------------------------------------------------------------------------------
@@ -353,82 +414,138 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    # step 0 is the exact first communication; then W warm-up steps; then K timed steps
+    def timed(run_step, count, per_step):
+        """`count` steps between two CUDA events on the launching stream (plus one event per step when
+        `per_step`), synchronised on both sides.  Returns (total ms, per-step ms or None, wall t0, wall t1)."""
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(count + 1 if per_step else 2)]
+        barrier()
+        t0 = time.time()
+        ev[0].record()
+        for k in range(count):
+            run_step(k)
+            if per_step:
+                ev[k + 1].record()
+        if not per_step:
+            ev[1].record()
+        torch.cuda.synchronize()
+        t1 = time.time()
+        each = [ev[k].elapsed_time(ev[k + 1]) for k in range(count)] if per_step else None
+        return ev[0].elapsed_time(ev[-1]), each, t0, t1
+
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
+    bytes_per_launch = algorithmic_bytes_per_coordinate(n, gb, pb, args.mode, args.kind) * d
+    peak, peak_kind = measured_hbm_peak()
+
+    def sustained_segment(run_step, ms_guess, seconds):
+        """At least `seconds` of steps back to back (no event between steps), with the clock sampled across it."""
+        count = max(20, int(math.ceil(seconds * 1e3 / max(ms_guess, 1e-3))))
+        ms, _, t0, t1 = timed(run_step, count, per_step=False)
+        ck = sampler.window(t0, t1)
+        per = ms / count
+        out = {"steps": count, "seconds": ms * 1e-3, "ms_per_step": per, "achieved": bytes_per_launch / (per * 1e-3) / 1e9,
+               "frac": bytes_per_launch / (per * 1e-3) / 1e9 / peak, "sm_mhz_median": ck["sm_mhz"],
+               "sm_mhz_min": ck.get("sm_mhz_min"), "power_w_max": ck["power_w_max"], "reasons": ck["reasons"],
+               "samples": ck["samples"]}
+        if ck["sm_mhz"]:
+            out["sm_clocks_per_worker_unit"] = per * 1e-3 * ck["sm_mhz"] * 1e6 * sms / (n * d / 4)
+        return out, count
+
+    # step 0 is the exact first communication; then W warm-up steps; then K timed steps; then the sustained segment
+    uuid = None
+    try:
+        uuid = str(torch.cuda.get_device_properties(device).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(local_rank, uuid)
+    sampler.start()
     step(0)
-    for k in range(1, 1 + max(args.warmup, 3)):
+    W = max(args.warmup, 3)
+    for k in range(1, 1 + W):
         step(k)
     barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     time.sleep(0.3)
     K = args.steps
-    events = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
     launches0 = lib.intsgd_launch_count()
-    barrier()
-    t_wall0 = time.time()
-    events[0].record()
-    for k in range(K):
-        step(1000 + k)
-        events[k + 1].record()
-    torch.cuda.synchronize()
-    t_wall1 = time.time()
+    total_ms, per_step_ms, t_wall0, t_wall1 = timed(lambda k: step(1000 + k), K, per_step=True)
     launches = lib.intsgd_launch_count() - launches0
-    barrier()
-    clocks = sampler.stop(t_wall0, t_wall1)
-    total_ms = events[0].elapsed_time(events[K])
-    per_step_ms = [events[k].elapsed_time(events[k + 1]) for k in range(K)]
+    clocks = sampler.window(t_wall0, t_wall1)
+    applied = 1 + W + K
+    sustained = None
+    if args.sustain_seconds > 0:
+        sustained, count = sustained_segment(lambda k: step(5000 + k), total_ms / K, args.sustain_seconds)
+        applied += count
     st = lib.intsgd_get_stats()   # raises if a step was refused (scale not finite) or a bounded wait expired
-    expected_steps = 1 + max(args.warmup, 3) + K
-    if st["step"] != expected_steps:
-        raise SystemExit(f"bench.py: {st['step']} steps were applied, {expected_steps} were enqueued: the timing is void")
+    if st["step"] != applied:
+        raise SystemExit(f"bench.py: {st['step']} steps were applied, {applied} were enqueued: the timing is void")
     total_ms = replicas.max_over_ranks(dist, total_ms, device)
     value = world * n * d * K / (total_ms * 1e-3)
-    bytes_per_launch = algorithmic_bytes_per_coordinate(n, gb, pb, args.mode, args.kind) * d
     avg_ms = statistics.mean(per_step_ms)
-    peak, peak_kind = measured_hbm_peak()
     achieved = bytes_per_launch / (avg_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic_per_launch(args, d), "peak_source": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
                 "algorithmic_bytes_per_launch": bytes_per_launch, "kernel_ms_avg": avg_ms,
                 "kernel_ms_median": statistics.median(per_step_ms),
-                "note": "per-step CUDA-event time (one-thread scale kernel + the vector kernel(s))"}
-    if clocks and clocks.get("sm_mhz"):
-        # The random-rounding kernel is co-limited by instruction issue (Philox): its time follows the SM clock.
-        # SM clocks spent per worker unit (4 gradient elements of one worker), from the clock sampled under load.
-        sms = torch.cuda.get_device_properties(device).multi_processor_count
+                "note": "per-step CUDA-event time of the K timed steps (one-thread scale kernel + the vector kernel(s)); "
+                        "`sustained` is the same step over a segment long enough for the board to settle at its power cap",
+                "sustained": sustained}
+    if clocks.get("sm_mhz"):
         roofline["sm_clocks_per_worker_unit"] = avg_ms * 1e-3 * clocks["sm_mhz"] * 1e6 * sms / (n * d / 4)
-        if roofline["traffic"] is not None:
-            # second limit: instruction issue (4 schedulers x 32 lanes per SM and clock, at the clock sampled under load)
-            ipe = NCU_TRAFFIC["instructions_per_element"]
-            issued = ipe * n * d / (avg_ms * 1e-3)
-            peak_issue = sms * 128 * clocks["sm_mhz"] * 1e6
-            roofline["co_limit"] = {"bound": "alu", "achieved": issued / 1e12, "peak": peak_issue / 1e12,
-                                    "unit": "T thread-instructions/s", "frac": issued / peak_issue,
-                                    "instructions_per_element": ipe,
-                                    "note": "instruction count from the ncu capture; peak = SMs x 128 lanes x sampled SM clock"}
 
-    # ---- the other rounding modes on the same buffers, short bursts (context for the headline; 1 GPU only) ----
+    # ---- second limit: the 32x32->64-bit multiplies of Philox4x32-10, against their rate measured alone ----
+    mults = wide_multiplies_per_worker_unit(args, n)
+    if mults > 0 and world == 1:
+        blocks_per_thread = 1 << 14
+        lib.intsgd_selftest_philox_rate(256, stream=stream)       # loads the kernel
+        nblocks = 0
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0 = time.time()
+        ev0.record()
+        for _ in range(6):
+            nblocks += lib.intsgd_selftest_philox_rate(blocks_per_thread, stream=stream)
+        ev1.record()
+        torch.cuda.synchronize()
+        t1 = time.time()
+        alone_ms = ev0.elapsed_time(ev1)
+        ck = sampler.window(t0, t1)
+        if ck["sm_mhz"]:
+            per_clock_alone = 16.0 * nblocks / (alone_ms * 1e-3 * ck["sm_mhz"] * 1e6 * sms)
+
+            def per_clock(ms, mhz):
+                return mults * (n * d / 4) / (ms * 1e-3 * mhz * 1e6 * sms)
+
+            co = {"bound": "alu", "unit": "32x32->64-bit products per SM clock and SM",
+                  "peak": per_clock_alone, "multiplies_per_worker_unit": mults,
+                  "peak_source": "rounds 3-10 of Philox4x32-10 alone (register-only kernel, 512 threads per SM, two chains "
+                                 f"per thread), {alone_ms:.0f} ms at {ck['sm_mhz']:.0f} MHz"}
+            if clocks.get("sm_mhz"):
+                co["achieved"] = per_clock(avg_ms, clocks["sm_mhz"])
+                co["frac"] = co["achieved"] / per_clock_alone
+            if sustained and sustained.get("sm_mhz_median"):
+                co["sustained_achieved"] = per_clock(sustained["ms_per_step"], sustained["sm_mhz_median"])
+                co["sustained_frac"] = co["sustained_achieved"] / per_clock_alone
+            roofline["co_limit"] = co
+
+    # ---- the other rounding modes on the same buffers (context for the headline; 1 GPU only): a burst each, and the
+    # comparison-form draw (the first reading of how Int(t) is drawn) through the same sustained segment ----
     variants = None
     if world == 1 and not args.no_variants and mode == pkg.MODE_FUSED and args.kind == "intsgd":
         variants = []
         names = {"random": pkg.ROUND_RANDOM, "compare": pkg.ROUND_RANDOM_COMPARE, "random16": pkg.ROUND_RANDOM16,
                  "nearest": pkg.ROUND_NEAREST}
         for name, rd in names.items():
+            time.sleep(0.5)
             with pkg.IntSGD(n, d, grad_dtype=grad_dtype, payload_dtype=payload_dtype, rounding=rd, seed=1, device=local_rank) as vlib:
+                vstep = lambda k: vlib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=mode, stream=stream)
                 vlib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=pkg.MODE_EXACT, stream=stream)
                 for _ in range(3):
-                    vlib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=mode, stream=stream)
-                ev = [torch.cuda.Event(enable_timing=True) for _ in range(31)]
-                torch.cuda.synchronize()
-                ev[0].record()
-                for k in range(30):
-                    vlib.intsgd_step(grads, x, agg, eta_k=args.eta, mode=mode, stream=stream)
-                    ev[k + 1].record()
-                torch.cuda.synchronize()
-                ms = statistics.median(ev[k].elapsed_time(ev[k + 1]) for k in range(30))
-            variants.append({"rounding": name, "burst_ms_median_of_30": ms,
-                             "hbm_frac": bytes_per_launch / (ms * 1e-3) / 1e9 / peak})
-            time.sleep(0.5)
+                    vstep(0)
+                _, each, _, _ = timed(vstep, 30, per_step=True)
+                ms = statistics.median(each)
+                entry = {"rounding": name, "burst_ms_median_of_30": ms, "hbm_frac": bytes_per_launch / (ms * 1e-3) / 1e9 / peak}
+                if name == "compare" and args.sustain_seconds > 0:
+                    entry["sustained"], _ = sustained_segment(vstep, ms, args.sustain_seconds)
+            variants.append(entry)
 
     # ---- end to end through the host-buffer entry point (rank-local; max over ranks) ----
     e2e = None
@@ -466,9 +583,10 @@ def main():
             except Exception as exc:   # a box that cannot spawn processes still reports the one-thread figure
                 cpu["all_cores"] = {"unavailable": repr(exc)}
 
+    sampler.stop()
     if rank == 0:
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if args.grad == "f32" else "bf16->f32", "data": "synthetic", "config": workload_config(args),
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,

@@ -234,6 +234,14 @@ int intsgd_set_fused_path(intsgd_ctx* ctx, int32_t path);
  * It touches no vector and no other state. */
 int intsgd_selftest_wait_expiry(intsgd_ctx* ctx, void* stream);
 
+/* Diagnostic for roofline reports: how fast this GPU gets through the integer arithmetic of the random stream
+ * when it does nothing else.  Enqueues one register-only kernel (one block of 512 threads per SM, no vector is
+ * touched) in which every thread computes blocks_per_thread (2 .. 2^24, rounded down to even) blocks of rounds
+ * 3-10 of Philox4x32-10 -- the per-worker part of a draw in the pipelined kernels, 16 32x32->64-bit products each --
+ * as two dependent chains.  *philox_blocks (may be NULL) receives the number of blocks the launch computes; the
+ * caller times the launch on `stream`.  The step kernels' random rounding cannot run faster than this rate. */
+int intsgd_selftest_philox_rate(intsgd_ctx* ctx, int64_t blocks_per_thread, int64_t* philox_blocks, void* stream);
+
 /* Number of kernels this library has launched on the context since creation. */
 int64_t intsgd_launch_count(const intsgd_ctx* ctx);
 

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "intsgd_diana.cuh"
+#include "intsgd_encode_pipe.cuh"
 #include "intsgd_kernels.cuh"
 #include "intsgd_pipe.cuh"
 
@@ -138,6 +139,7 @@ void base_params(const intsgd_ctx* ctx, VecParams& P) {
     P.Lf = ctx->Lf;
     P.agg_limit = (ctx->cfg.payload_dtype == INTSGD_PAYLOAD_I8) ? 127 : std::numeric_limits<int32_t>::max();
     P.keys = ctx->keys;
+    P.tab = ctx->tab;
 }
 
 int check_vector(intsgd_ctx* ctx, const void* p, size_t elem, const char* what, bool* all16) {
@@ -207,7 +209,34 @@ void launch_encode_a(const intsgd_ctx* ctx, const VecParams& P, dim3 grid, bool 
     if (aligned) launch_encode_r<GRAD, PAY, true>(ctx, P, grid, s);
     else launch_encode_r<GRAD, PAY, false>(ctx, P, grid, s);
 }
+int launch_encode_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s);
+bool pipe_eligible(const intsgd_ctx* ctx, bool aligned, int64_t d);
+void fill_block_params(const intsgd_ctx* ctx, VecParams& P, int64_t covered_end);
+
+template <int GRAD, int PAY, bool ALIGNED>
+void launch_encode_blocks_r(const intsgd_ctx* ctx, const VecParams& P, dim3 grid, cudaStream_t s) {
+    switch (ctx->cfg.rounding) {
+        case INTSGD_ROUND_NEAREST: encode_blocks_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_NEAREST><<<grid, ctx->threads, 0, s>>>(P); break;
+        case INTSGD_ROUND_RANDOM16: encode_blocks_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_RANDOM16><<<grid, ctx->threads, 0, s>>>(P); break;
+        case INTSGD_ROUND_RANDOM_COMPARE: encode_blocks_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_RANDOM_COMPARE><<<grid, ctx->threads, 0, s>>>(P); break;
+        default: encode_blocks_kernel<GRAD, PAY, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P); break;
+    }
+}
+template <int GRAD, int PAY>
+void launch_encode_blocks_a(const intsgd_ctx* ctx, const VecParams& P, dim3 grid, bool aligned, cudaStream_t s) {
+    if (aligned) launch_encode_blocks_r<GRAD, PAY, true>(ctx, P, grid, s);
+    else launch_encode_blocks_r<GRAD, PAY, false>(ctx, P, grid, s);
+}
+void launch_encode_blocks(const intsgd_ctx* ctx, const VecParams& P, dim3 grid, bool bf16, bool i8, bool aligned, cudaStream_t s) {
+    if (!bf16 && !i8) launch_encode_blocks_a<INTSGD_GRAD_F32, INTSGD_PAYLOAD_I32>(ctx, P, grid, aligned, s);
+    else if (!bf16) launch_encode_blocks_a<INTSGD_GRAD_F32, INTSGD_PAYLOAD_I8>(ctx, P, grid, aligned, s);
+    else if (!i8) launch_encode_blocks_a<INTSGD_GRAD_BF16, INTSGD_PAYLOAD_I32>(ctx, P, grid, aligned, s);
+    else launch_encode_blocks_a<INTSGD_GRAD_BF16, INTSGD_PAYLOAD_I8>(ctx, P, grid, aligned, s);
+}
+
 int launch_encode(intsgd_ctx* ctx, const VecParams& P, int workers, bool aligned, cudaStream_t s) {
+    // All the workers of a step in one launch: the pipelined kernel (a thread keeps its units across workers).
+    if (workers >= 2 && ctx->fused_path != 1 && pipe_eligible(ctx, aligned, P.d)) return launch_encode_pipe(ctx, P, s);
     dim3 grid((unsigned)grid_for(ctx, (ctx->cfg.d + 3) / 4), (unsigned)workers, 1);
     // spread the block budget over the workers handled by one launch
     if (workers > 1) {
@@ -216,6 +245,12 @@ int launch_encode(intsgd_ctx* ctx, const VecParams& P, int workers, bool aligned
         if ((int)grid.x > per) grid.x = (unsigned)per;
     }
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16, i8 = ctx->cfg.payload_dtype == INTSGD_PAYLOAD_I8;
+    if (ctx->bs.B > 0) {
+        VecParams Q = P;
+        fill_block_params(ctx, Q, (ctx->cfg.d >> 2) << 2);
+        launch_encode_blocks(ctx, Q, grid, bf16, i8, aligned, s);
+        return after_launch(ctx, "encode_blocks_kernel");
+    }
     if (!bf16 && !i8) launch_encode_a<INTSGD_GRAD_F32, INTSGD_PAYLOAD_I32>(ctx, P, grid, aligned, s);
     else if (!bf16 && i8) launch_encode_a<INTSGD_GRAD_F32, INTSGD_PAYLOAD_I8>(ctx, P, grid, aligned, s);
     else if (bf16 && !i8) launch_encode_a<INTSGD_GRAD_BF16, INTSGD_PAYLOAD_I32>(ctx, P, grid, aligned, s);
@@ -223,8 +258,27 @@ int launch_encode(intsgd_ctx* ctx, const VecParams& P, int workers, bool aligned
     return after_launch(ctx, "encode_kernel");
 }
 
+int launch_block_norm(intsgd_ctx* ctx, int64_t covered_end, bool check_status, bool advance_step, cudaStream_t s);
+
 int launch_aggregate(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t s) {
     const bool i8 = ctx->cfg.payload_dtype == INTSGD_PAYLOAD_I8;
+    if (ctx->bs.B > 0) {
+        VecParams Q = P;
+        const int64_t covered = (ctx->cfg.d >> 2) << 2;
+        fill_block_params(ctx, Q, covered);
+        // the step's scale kernel has cleared the edge partials; clearing them again here keeps a repeated
+        // aggregate (without a scale in between) correct as well
+        if (cudaMemsetAsync(ctx->bs.edge_sum, 0, sizeof(double) * ctx->bs.B, s) != cudaSuccess)
+            return fail(ctx, INTSGD_ERR_CUDA, "cudaMemsetAsync failed");
+        const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
+        if (!i8 && aligned) aggregate_blocks_kernel<INTSGD_PAYLOAD_I32, true><<<grid, ctx->threads, 0, s>>>(Q);
+        else if (!i8) aggregate_blocks_kernel<INTSGD_PAYLOAD_I32, false><<<grid, ctx->threads, 0, s>>>(Q);
+        else if (aligned) aggregate_blocks_kernel<INTSGD_PAYLOAD_I8, true><<<grid, ctx->threads, 0, s>>>(Q);
+        else aggregate_blocks_kernel<INTSGD_PAYLOAD_I8, false><<<grid, ctx->threads, 0, s>>>(Q);
+        const int rc = after_launch(ctx, "aggregate_blocks_kernel");
+        if (rc != INTSGD_OK) return rc;
+        return launch_block_norm(ctx, covered, true, true, s);
+    }
     const int64_t items = (i8 && aligned) ? (ctx->cfg.d + 15) / 16 : (i8 ? ctx->cfg.d : (ctx->cfg.d + 3) / 4);
     const int grid = grid_for(ctx, items);
     if (!i8 && aligned) aggregate_kernel<INTSGD_PAYLOAD_I32, true><<<grid, ctx->threads, 0, s>>>(P);
@@ -303,6 +357,69 @@ bool pipe_eligible(const intsgd_ctx* ctx, bool aligned, int64_t d) {
     return aligned && ctx->cfg.d <= ((int64_t)1 << 34) && units >= 2;
 }
 
+// Pipelined encode: the default ring shape of the fused kernel (512 consumers, 2 units each, 3 stages of 4 fp32
+// or 8 bf16 worker tiles).
+template <int GRAD, int PAY, int ROUND, bool BLOCKS>
+cudaError_t launch_encode_pipe_b(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
+    constexpr int NC = 512, UPT = 2, NS = 3, G = (GRAD == INTSGD_GRAD_BF16) ? 8 : 4;
+    auto kernel = encode_pipe_kernel<GRAD, PAY, ROUND, BLOCKS, NC, UPT, G, NS>;
+    const int smem = NS * G * NC * UPT * ((GRAD == INTSGD_GRAD_F32) ? 16 : 8);
+    static std::atomic<bool> configured[kMaxDevices] = {};
+    const int dev = ctx->cfg.device;
+    if (dev < 0 || dev >= kMaxDevices || !configured[dev].load(std::memory_order_acquire)) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < kMaxDevices) configured[dev].store(true, std::memory_order_release);
+    }
+    PP.tiles = (PP.units + NC * UPT - 1) / (NC * UPT);
+    const int64_t grid = PP.tiles < ctx->sm_count ? PP.tiles : ctx->sm_count;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(NC + 32, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->follows_scale ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, PP);
+}
+template <int GRAD, int PAY, int ROUND>
+cudaError_t launch_encode_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
+    return ctx->bs.B > 0 ? launch_encode_pipe_b<GRAD, PAY, ROUND, true>(ctx, PP, s) : launch_encode_pipe_b<GRAD, PAY, ROUND, false>(ctx, PP, s);
+}
+template <int GRAD, int PAY>
+cudaError_t launch_encode_pipe_r(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
+    switch (ctx->cfg.rounding) {
+        case INTSGD_ROUND_NEAREST: return launch_encode_pipe_t<GRAD, PAY, INTSGD_ROUND_NEAREST>(ctx, PP, s);
+        case INTSGD_ROUND_RANDOM16: return launch_encode_pipe_t<GRAD, PAY, INTSGD_ROUND_RANDOM16>(ctx, PP, s);
+        case INTSGD_ROUND_RANDOM_COMPARE: return launch_encode_pipe_t<GRAD, PAY, INTSGD_ROUND_RANDOM_COMPARE>(ctx, PP, s);
+        default: return launch_encode_pipe_t<GRAD, PAY, INTSGD_ROUND_RANDOM>(ctx, PP, s);
+    }
+}
+int launch_encode_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
+    PipeParams PP;
+    PP.v = P;
+    const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16, i8 = ctx->cfg.payload_dtype == INTSGD_PAYLOAD_I8;
+    int64_t units = P.d >> 2;
+    if (bf16) units &= ~(int64_t)1;   // bulk copies move multiples of 16 bytes
+    PP.units = units;
+    PP.tiles = 0;
+    PP.fast_limit = ctx->Lf;   // not used: out-of-range values take the counting rule on the spot
+    if (ctx->bs.B > 0) fill_block_params(ctx, PP.v, units << 2);
+    cudaError_t e;
+    if (!bf16 && !i8) e = launch_encode_pipe_r<INTSGD_GRAD_F32, INTSGD_PAYLOAD_I32>(ctx, PP, s);
+    else if (!bf16) e = launch_encode_pipe_r<INTSGD_GRAD_F32, INTSGD_PAYLOAD_I8>(ctx, PP, s);
+    else if (!i8) e = launch_encode_pipe_r<INTSGD_GRAD_BF16, INTSGD_PAYLOAD_I32>(ctx, PP, s);
+    else e = launch_encode_pipe_r<INTSGD_GRAD_BF16, INTSGD_PAYLOAD_I8>(ctx, PP, s);
+    if (e != cudaSuccess) {
+        std::snprintf(ctx->err, 256, "encode_pipe_kernel launch failed: %s", cudaGetErrorString(e));
+        return INTSGD_ERR_CUDA;
+    }
+    return after_launch(ctx, "encode_pipe_kernel");
+}
+
 void fill_block_params(const intsgd_ctx* ctx, VecParams& P, int64_t covered_end) {
     P.bp.offsets = ctx->bs.offsets;
     P.bp.alpha = ctx->bs.alpha;
@@ -316,7 +433,7 @@ void fill_block_params(const intsgd_ctx* ctx, VecParams& P, int64_t covered_end)
 }
 
 // Finishes a block-wise step: per-segment squared step lengths, total, step counter.
-int launch_block_norm(intsgd_ctx* ctx, int64_t covered_end, bool check_status, cudaStream_t s) {
+int launch_block_norm(intsgd_ctx* ctx, int64_t covered_end, bool check_status, bool advance_step, cudaStream_t s) {
     const NormPlan& plan = (ctx->plan[0].covered_end == covered_end) ? ctx->plan[0] : ctx->plan[1];
     if (plan.covered_end != covered_end) return fail(ctx, INTSGD_ERR_CUDA, "internal: no reduction plan for this launch");
     if (plan.num_slices > 0) {
@@ -324,20 +441,21 @@ int launch_block_norm(intsgd_ctx* ctx, int64_t covered_end, bool check_status, c
         const int rc = after_launch(ctx, "block_norm_slices_kernel");
         if (rc != INTSGD_OK) return rc;
     }
-    block_norm_kernel<<<ctx->bs.B, 128, 0, s>>>(ctx->d_state, ctx->bs, plan, ctx->cfg.d, check_status ? 1 : 0);
+    block_norm_kernel<<<ctx->bs.B, 128, 0, s>>>(ctx->d_state, ctx->bs, plan, ctx->cfg.d, check_status ? 1 : 0,
+                                                advance_step ? 1 : 0);
     return after_launch(ctx, "block_norm_kernel");
 }
 
 int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     PipeParams PP;
     PP.v = P;
-    PP.tab = ctx->tab;
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
     int64_t units = P.d >> 2;
     if (bf16) units &= ~(int64_t)1;   // bulk copies move multiples of 16 bytes
     PP.units = units;
     PP.tiles = 0;   // set by the launcher from the tile shape
-    if (ctx->bs.B > 0) fill_block_params(ctx, PP.v, units << 2);
+    const int64_t covered_end = (P.unit_base << 2) + (units << 2);   // in coordinates of the whole vector
+    if (ctx->bs.B > 0) fill_block_params(ctx, PP.v, covered_end);
     // Rounded values are summed as integer-valued floats: exact while n * (T + 1) <= 2^24.
     const float t_max = (float)((1 << 24) / ctx->cfg.n - 2);
     PP.fast_limit = ctx->Lf < t_max ? ctx->Lf : t_max;
@@ -357,7 +475,8 @@ int launch_fused_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     }
     const int rc = after_launch(ctx, "fused_pipe_kernel");
     if (rc != INTSGD_OK || ctx->bs.B == 0) return rc;
-    return launch_block_norm(ctx, units << 2, true, s);
+    if (P.window_flags & kWindowHoldStep) return rc;   // the per-segment norms are finished after the step's last window
+    return launch_block_norm(ctx, covered_end, true, true, s);
 }
 
 template <int GRAD, bool ALIGNED>
@@ -379,15 +498,15 @@ int launch_fused(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
     if (ctx->bs.B > 0) {
         VecParams Q = P;
-        const int64_t covered = (ctx->cfg.d >> 2) << 2;
+        const int64_t covered = (P.unit_base << 2) + ((P.d >> 2) << 2);
         fill_block_params(ctx, Q, covered);
         if (!bf16 && aligned) launch_fused_blocks_r<INTSGD_GRAD_F32, true>(ctx, Q, grid, s);
         else if (!bf16) launch_fused_blocks_r<INTSGD_GRAD_F32, false>(ctx, Q, grid, s);
         else if (aligned) launch_fused_blocks_r<INTSGD_GRAD_BF16, true>(ctx, Q, grid, s);
         else launch_fused_blocks_r<INTSGD_GRAD_BF16, false>(ctx, Q, grid, s);
         const int rc = after_launch(ctx, "fused_step_blocks_kernel");
-        if (rc != INTSGD_OK) return rc;
-        return launch_block_norm(ctx, covered, true, s);
+        if (rc != INTSGD_OK || (P.window_flags & kWindowHoldStep)) return rc;
+        return launch_block_norm(ctx, covered, true, true, s);
     }
     if (!bf16 && aligned) launch_fused_r<INTSGD_GRAD_F32, true>(ctx, P, grid, s);
     else if (!bf16) launch_fused_r<INTSGD_GRAD_F32, false>(ctx, P, grid, s);
@@ -446,7 +565,6 @@ cudaError_t launch_diana_pipe_r(const intsgd_ctx* ctx, PipeParams& PP, cudaStrea
 int launch_diana_pipe(intsgd_ctx* ctx, const VecParams& P, cudaStream_t s) {
     PipeParams PP;
     PP.v = P;
-    PP.tab = ctx->tab;
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
     int64_t units = P.d >> 2;
     if (bf16) units &= ~(int64_t)1;   // bulk copies move multiples of 16 bytes
@@ -477,17 +595,18 @@ int launch_exact(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStream_t
     const bool bf16 = ctx->cfg.grad_dtype == INTSGD_GRAD_BF16;
     if (ctx->bs.B > 0) {
         VecParams Q = P;
-        const int64_t covered = (ctx->cfg.d >> 2) << 2;
+        const int64_t covered = (P.unit_base << 2) + ((P.d >> 2) << 2);
         fill_block_params(ctx, Q, covered);
-        if (cudaMemsetAsync(ctx->bs.edge_sum, 0, sizeof(double) * ctx->bs.B, s) != cudaSuccess)
+        if (!(P.window_flags & kWindowAccumulate) &&   // the first (or only) window of the step opens the edge partials
+            cudaMemsetAsync(ctx->bs.edge_sum, 0, sizeof(double) * ctx->bs.B, s) != cudaSuccess)
             return fail(ctx, INTSGD_ERR_CUDA, "cudaMemsetAsync failed");
         if (!bf16 && aligned) exact_step_blocks_kernel<INTSGD_GRAD_F32, true><<<grid, ctx->threads, 0, s>>>(Q);
         else if (!bf16) exact_step_blocks_kernel<INTSGD_GRAD_F32, false><<<grid, ctx->threads, 0, s>>>(Q);
         else if (aligned) exact_step_blocks_kernel<INTSGD_GRAD_BF16, true><<<grid, ctx->threads, 0, s>>>(Q);
         else exact_step_blocks_kernel<INTSGD_GRAD_BF16, false><<<grid, ctx->threads, 0, s>>>(Q);
         const int rc = after_launch(ctx, "exact_step_blocks_kernel");
-        if (rc != INTSGD_OK) return rc;
-        return launch_block_norm(ctx, covered, false, s);
+        if (rc != INTSGD_OK || (P.window_flags & kWindowHoldStep)) return rc;
+        return launch_block_norm(ctx, covered, false, true, s);
     }
     if (!bf16 && aligned) exact_step_kernel<INTSGD_GRAD_F32, true><<<grid, ctx->threads, 0, s>>>(P);
     else if (!bf16) exact_step_kernel<INTSGD_GRAD_F32, false><<<grid, ctx->threads, 0, s>>>(P);
@@ -672,7 +791,6 @@ int intsgd_scale(intsgd_ctx* ctx, double eta_k, double dx2_override, void* strea
 int intsgd_sqdiff(intsgd_ctx* ctx, const float* x, const float* x_prev, void* stream) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
-    if (ctx->bs.B > 0) return block_mode_unsupported(ctx, "intsgd_sqdiff");
     bool al = true;
     int rc;
     if ((rc = check_vector(ctx, x, 4, "x", &al)) != INTSGD_OK) return rc;
@@ -684,6 +802,15 @@ int intsgd_sqdiff(intsgd_ctx* ctx, const float* x, const float* x_prev, void* st
     cudaStream_t s = (cudaStream_t)stream;
     ctx->last_stream = s;
     const int grid = grid_for(ctx, (ctx->cfg.d + 3) / 4);
+    if (ctx->bs.B > 0) {   // one squared difference per block (Algorithm 2's moving averages are per block)
+        const int64_t covered = (ctx->cfg.d >> 2) << 2;
+        fill_block_params(ctx, P, covered);
+        CUDA_TRY(ctx, cudaMemsetAsync(ctx->bs.edge_sum, 0, sizeof(double) * ctx->bs.B, s));
+        if (al) sqdiff_blocks_kernel<true><<<grid, ctx->threads, 0, s>>>(P);
+        else sqdiff_blocks_kernel<false><<<grid, ctx->threads, 0, s>>>(P);
+        if ((rc = after_launch(ctx, "sqdiff_blocks_kernel")) != INTSGD_OK) return rc;
+        return launch_block_norm(ctx, covered, false, false, s);
+    }
     if (al) sqdiff_kernel<true><<<grid, ctx->threads, 0, s>>>(P);
     else sqdiff_kernel<false><<<grid, ctx->threads, 0, s>>>(P);
     return after_launch(ctx, "sqdiff_kernel");
@@ -693,7 +820,8 @@ int intsgd_encode(intsgd_ctx* ctx, int32_t worker, const void* grad, void* paylo
                   void* stream) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
-    if (ctx->bs.B > 0) return block_mode_unsupported(ctx, "intsgd_encode");
+    if (ctx->bs.B > 0 && alpha_override == alpha_override)
+        return fail(ctx, INTSGD_ERR_UNSUPPORTED, "alpha_override is not available with block-wise scales (pass NaN)");
     if (worker < 0 || worker >= ctx->cfg.n) return fail(ctx, INTSGD_ERR_INVALID_ARG, "worker index out of range");
     if (std::isinf(alpha_override) || alpha_override <= 0.0f)
         return fail(ctx, INTSGD_ERR_INVALID_ARG, "alpha_override must be NaN (use state) or finite and > 0");
@@ -714,7 +842,6 @@ int intsgd_encode(intsgd_ctx* ctx, int32_t worker, const void* grad, void* paylo
 int intsgd_aggregate(intsgd_ctx* ctx, const void* const* payloads, float* x, int32_t* agg, void* stream) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
-    if (ctx->bs.B > 0) return block_mode_unsupported(ctx, "intsgd_aggregate");
     if (!payloads) return fail(ctx, INTSGD_ERR_INVALID_ARG, "payloads is NULL");
     bool al = true;
     int rc;
@@ -739,7 +866,6 @@ int intsgd_step(intsgd_ctx* ctx, const void* const* grads, void* const* payload_
     if (mode != INTSGD_MODE_EXACT && mode != INTSGD_MODE_TWO_KERNEL && mode != INTSGD_MODE_FUSED)
         return fail(ctx, INTSGD_ERR_INVALID_ARG, "bad mode");
     if (!grads) return fail(ctx, INTSGD_ERR_INVALID_ARG, "grads is NULL");
-    if (mode == INTSGD_MODE_TWO_KERNEL && ctx->bs.B > 0) return block_mode_unsupported(ctx, "INTSGD_MODE_TWO_KERNEL");
     if (mode == INTSGD_MODE_TWO_KERNEL && !payload_scratch)
         return fail(ctx, INTSGD_ERR_INVALID_ARG, "TWO_KERNEL mode needs payload_scratch");
     if (!(eta_k > 0.0) || !std::isfinite(eta_k)) return fail(ctx, INTSGD_ERR_INVALID_ARG, "eta_k must be finite and > 0");
@@ -780,7 +906,10 @@ int intsgd_step(intsgd_ctx* ctx, const void* const* grads, void* const* payload_
     }
     if ((rc = launch_scale(ctx, eta_k, -1.0, s)) != INTSGD_OK) return rc;
     P.worker_base = 0;
-    if ((rc = launch_encode(ctx, P, ctx->cfg.n, al_enc, s)) != INTSGD_OK) return rc;
+    ctx->follows_scale = true;
+    rc = launch_encode(ctx, P, ctx->cfg.n, al_enc, s);
+    ctx->follows_scale = false;
+    if (rc != INTSGD_OK) return rc;
     VecParams A;
     base_params(ctx, A);
     for (int i = 0; i < ctx->cfg.n; ++i) A.in[i] = payload_scratch[i];
@@ -947,7 +1076,7 @@ int intsgd_step_host(intsgd_ctx* ctx, const void* const* host_grads, float* host
         }
     }
     cudaStream_t s = (cudaStream_t)stream;
-    if (d > (size_t)kHostWindow && ctx->bs.B == 0) {
+    if (d > (size_t)kHostWindow) {
         const int rc = step_host_windowed(ctx, host_grads, host_x, host_agg, eta_k, mode, s);
         if (rc != INTSGD_OK) return rc;
         CUDA_TRY(ctx, cudaStreamSynchronize(ctx->back_stream));
@@ -998,6 +1127,20 @@ int intsgd_selftest_wait_expiry(intsgd_ctx* ctx, void* stream) {
     ctx->last_stream = s;
     wait_expiry_kernel<<<1, 32, 0, s>>>(ctx->d_state, 64u);
     return after_launch(ctx, "wait_expiry_kernel");
+}
+
+int intsgd_selftest_philox_rate(intsgd_ctx* ctx, int64_t blocks_per_thread, int64_t* philox_blocks, void* stream) {
+    if (!ctx) return INTSGD_ERR_INVALID_ARG;
+    if (blocks_per_thread < 2 || blocks_per_thread > ((int64_t)1 << 24))
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "blocks_per_thread must be in 2..2^24");
+    DeviceGuard guard(ctx->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    ctx->last_stream = s;
+    const uint32_t per_chain = (uint32_t)(blocks_per_thread / 2);
+    // the sink is the state block's spare word; the kernel's store condition never holds in practice
+    philox_rate_kernel<<<ctx->sm_count, 512, 0, s>>>(ctx->keys, per_chain, &ctx->d_state->pad2);
+    if (philox_blocks) *philox_blocks = (int64_t)ctx->sm_count * 512 * 2 * per_chain;
+    return after_launch(ctx, "philox_rate_kernel");
 }
 
 int intsgd_get_state(intsgd_ctx* ctx, intsgd_state* out) {

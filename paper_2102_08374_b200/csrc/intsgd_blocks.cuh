@@ -215,9 +215,9 @@ __global__ void __launch_bounds__(256) block_norm_slices_kernel(const DevState* 
 
 // Pass 2: thread block l adds the slices of segment l in order, then the (at most two) edge partials
 // and the segment's tail coordinates.  The block that finishes last adds the B results into
-// state.dx2 and advances the step counter.
+// state.dx2 and (after a step, not after intsgd_sqdiff) advances the step counter.
 __global__ void __launch_bounds__(128) block_norm_kernel(DevState* st, BlockState bs, NormPlan plan, int64_t d,
-                                                         int32_t check_status) {
+                                                         int32_t check_status, int32_t advance_step) {
     __shared__ double s_warp[32];
     __shared__ bool s_last;
     if (check_status && st->status != INTSGD_OK) return;
@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(128) block_norm_kernel(DevState* st, BlockStat
     const double sum = block_tree(w2, s_warp);
     if (threadIdx.x == 0) {
         st->dx2 = sum;
-        st->step += 1;
+        if (advance_step) st->step += 1;
         st->ticket = 0;
     }
 }
@@ -290,23 +290,239 @@ __global__ void __launch_bounds__(512) fused_step_blocks_kernel(const __grid_con
 
     const int64_t full = P.d >> 2;   // == bp.covered_end / 4
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    // A launch may cover a window of the vector: `unit` indexes the launch's pointers, `unit + P.unit_base` the
+    // whole vector (partition tables, chunk partials, random stream).
     for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x - lane); base < full; base += stride) {
-        const int64_t unit = base + lane;
+        const int64_t unit = base + lane, gunit = unit + P.unit_base;
         const bool active = unit < full;
         int s_lo, s_hi;
-        chunk_segments(bp, base, s_lo, s_hi);
+        chunk_segments(bp, base + P.unit_base, s_lo, s_hi);
         double sq[4] = {0.0, 0.0, 0.0, 0.0};
         int seg[4] = {-1, -1, -1, -1};
         if (active) {
-            const UnitScale us = unit_scale(bp, unit, s_lo, s_hi);
+            const UnitScale us = unit_scale(bp, gunit, s_lo, s_hi);
             int4 S = make_int4(0, 0, 0, 0);
+            PhiloxThreadPart tp = {0u, 0u, 0u};   // the unit's half of Philox rounds 1-2 serves all n workers
+            if (ROUND != INTSGD_ROUND_NEAREST) tp = draw_thread_part<ROUND>(gunit, step, P.keys);
 #pragma unroll 4
             for (int i = 0; i < n; ++i) {
                 const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
                 uint4 w = make_uint4(0, 0, 0, 0);
-                if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, (uint32_t)i, step, P.keys);
+                if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit_folded<ROUND>(tp, gunit, P.tab.e[i], (uint32_t)i, step, P.keys);
                 const int4 q = round_unit_scaled<ROUND>(gv, us.a01, us.a23, w, P.Lf, &s_cnt[i], nonf_slot);
                 S.x += q.x; S.y += q.y; S.z += q.z; S.w += q.w;
+            }
+            const float4 xo = load_f4<ALIGNED>(P.x, unit);
+            float4 xn;
+            xn.x = update_coord_sq(xo.x, __int2float_rn(S.x), us.c.x, sq[0]);
+            xn.y = update_coord_sq(xo.y, __int2float_rn(S.y), us.c.y, sq[1]);
+            xn.z = update_coord_sq(xo.z, __int2float_rn(S.z), us.c.z, sq[2]);
+            xn.w = update_coord_sq(xo.w, __int2float_rn(S.w), us.c.w, sq[3]);
+            store_f4<ALIGNED>(P.x, unit, xn);
+            if (P.agg) store_i4<ALIGNED>(P.agg, unit, S);
+            note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
+            note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
+        }
+        chunk_commit(bp, base + P.unit_base, s_lo, s_hi, sq, seg);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t j = full << 2; j < P.d; ++j) {
+            const int64_t gj = j + (P.unit_base << 2);
+            float alpha, c;
+            coord_scale(bp, gj, alpha, c);
+            int S = 0;
+            for (int i = 0; i < n; ++i) {
+                uint32_t word = 0;
+                if (ROUND != INTSGD_ROUND_NEAREST) {
+                    const uint4 w4 = draw_unit<ROUND>(gj >> 2, (uint32_t)i, step, P.keys);
+                    const uint32_t wv[4] = {w4.x, w4.y, w4.z, w4.w};
+                    word = wv[j & 3];
+                }
+                const float y = __fmul_rn(alpha, grad_at<GRAD>(P.in[i], j));
+                S += round_checked<ROUND>(y, word, P.Lf, &s_cnt[i], nonf_slot);
+            }
+            double sqj;
+            P.x[j] = update_coord_sq(P.x[j], __int2float_rn(S), c, sqj);
+            if (P.agg) P.agg[j] = S;
+            note_sum(S, P.agg_limit, acc);
+            bp.tail_sq[gj - bp.covered_end] = sqj;
+        }
+    }
+    counters_flush(s_cnt, st);
+    flush_sum_counters(acc, st);
+}
+
+// Exact first step with per-segment squared step lengths (Algorithm 2's Input line: x^1 is the
+// uncompressed mean step; its block norms start the moving averages).
+template <int GRAD, bool ALIGNED>
+__global__ void __launch_bounds__(512) exact_step_blocks_kernel(const __grid_constant__ VecParams P) {
+    const BlockParams& bp = P.bp;
+    const int n = P.n;
+    const float c0 = P.c_exact;
+    const int lane = threadIdx.x & 31;
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x - lane); base < full; base += stride) {
+        const int64_t unit = base + lane;
+        const bool active = unit < full;
+        int s_lo, s_hi;
+        chunk_segments(bp, base + P.unit_base, s_lo, s_hi);
+        double sq[4] = {0.0, 0.0, 0.0, 0.0};
+        int seg[4] = {-1, -1, -1, -1};
+        if (active) {
+            float4 m = load_grad4<GRAD, ALIGNED>(P.in[0], unit);
+#pragma unroll 4
+            for (int i = 1; i < n; ++i) {
+                const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
+                m.x = __fadd_rn(m.x, gv.x); m.y = __fadd_rn(m.y, gv.y);
+                m.z = __fadd_rn(m.z, gv.z); m.w = __fadd_rn(m.w, gv.w);
+            }
+            const float4 xo = load_f4<ALIGNED>(P.x, unit);
+            float4 xn;
+            xn.x = update_coord_sq(xo.x, m.x, c0, sq[0]);
+            xn.y = update_coord_sq(xo.y, m.y, c0, sq[1]);
+            xn.z = update_coord_sq(xo.z, m.z, c0, sq[2]);
+            xn.w = update_coord_sq(xo.w, m.w, c0, sq[3]);
+            store_f4<ALIGNED>(P.x, unit, xn);
+            if (s_lo == s_hi) {
+                seg[0] = seg[1] = seg[2] = seg[3] = s_lo;
+            } else {
+                const UnitScale us = unit_scale(bp, unit + P.unit_base, s_lo, s_hi);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
+            }
+        }
+        chunk_commit(bp, base + P.unit_base, s_lo, s_hi, sq, seg);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t j = full << 2; j < P.d; ++j) {
+            float m = grad_at<GRAD>(P.in[0], j);
+            for (int i = 1; i < n; ++i) m = __fadd_rn(m, grad_at<GRAD>(P.in[i], j));
+            double sqj;
+            P.x[j] = update_coord_sq(P.x[j], m, c0, sqj);
+            bp.tail_sq[j + (P.unit_base << 2) - bp.covered_end] = sqj;
+        }
+    }
+}
+
+// Per-segment ||x - x_prev||^2 for a caller that holds two iterates (the block-wise form of intsgd_sqdiff):
+// fp32 differences, exact squares, the same chunk partials and fixed-order sums as a step.
+template <bool ALIGNED>
+__global__ void __launch_bounds__(512) sqdiff_blocks_kernel(const __grid_constant__ VecParams P) {
+    const BlockParams& bp = P.bp;
+    const int lane = threadIdx.x & 31;
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x - lane); base < full; base += stride) {
+        const int64_t unit = base + lane;
+        int s_lo, s_hi;
+        chunk_segments(bp, base, s_lo, s_hi);
+        double sq[4] = {0.0, 0.0, 0.0, 0.0};
+        int seg[4] = {-1, -1, -1, -1};
+        if (unit < full) {
+            const float4 a = load_f4<ALIGNED>(P.x, unit), b = load_f4<ALIGNED>(P.x_prev, unit);
+            const float d0 = __fsub_rn(a.x, b.x), d1 = __fsub_rn(a.y, b.y), d2 = __fsub_rn(a.z, b.z), d3 = __fsub_rn(a.w, b.w);
+            sq[0] = (double)d0 * (double)d0; sq[1] = (double)d1 * (double)d1;
+            sq[2] = (double)d2 * (double)d2; sq[3] = (double)d3 * (double)d3;
+            if (s_lo == s_hi) {
+                seg[0] = seg[1] = seg[2] = seg[3] = s_lo;
+            } else {
+                const UnitScale us = unit_scale(bp, unit, s_lo, s_hi);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
+            }
+        }
+        chunk_commit(bp, base, s_lo, s_hi, sq, seg);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int64_t j = full << 2; j < P.d; ++j) {
+            const float dj = __fsub_rn(P.x[j], P.x_prev[j]);
+            bp.tail_sq[j - bp.covered_end] = (double)dj * (double)dj;
+        }
+    }
+}
+
+// Encode with block-wise scales, direct form (one worker per blockIdx.y): payload = clip(Int(alpha_l g)) with
+// the scale of the block each coordinate lies in (Algorithm 2's Int(alpha_{k,l} o g)).
+template <int GRAD, int PAY, bool ALIGNED, int ROUND>
+__global__ void __launch_bounds__(512) encode_blocks_kernel(const __grid_constant__ VecParams P) {
+    __shared__ cnt_t s_cnt[INTSGD_MAX_WORKERS + 1];
+    DevState* st = P.st;
+    if (st->status != INTSGD_OK) return;
+    counters_init(s_cnt);
+    const BlockParams& bp = P.bp;
+    const uint32_t step = st->step;
+    const int slot = blockIdx.y;
+    const uint32_t worker = (uint32_t)(P.worker_base + slot);
+    const void* g = P.in[slot];
+    void* out = P.out[slot];
+    cnt_t* clip_slot = &s_cnt[worker];
+    cnt_t* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
+    const uint4 e = P.tab.e[worker];
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
+        int s_lo, s_hi;
+        chunk_segments(bp, unit & ~(int64_t)31, s_lo, s_hi);
+        const UnitScale us = unit_scale(bp, unit, s_lo, s_hi);
+        const float4 gv = load_grad4<GRAD, ALIGNED>(g, unit);
+        uint4 w = make_uint4(0, 0, 0, 0);
+        if (ROUND != INTSGD_ROUND_NEAREST)
+            w = draw_unit_folded<ROUND>(draw_thread_part<ROUND>(unit, step, P.keys), unit, e, worker, step, P.keys);
+        store_payload4<PAY>(out, unit, round_unit_scaled<ROUND>(gv, us.a01, us.a23, w, P.Lf, clip_slot, nonf_slot), ALIGNED);
+    }
+    const int tail = (int)(P.d & 3);
+    if (tail && blockIdx.x == 0 && threadIdx.x == 0) {
+        uint4 w = make_uint4(0, 0, 0, 0);
+        if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(full, worker, step, P.keys);
+        const uint32_t wv[4] = {w.x, w.y, w.z, w.w};
+        for (int t = 0; t < tail; ++t) {
+            const int64_t j = 4 * full + t;
+            float alpha, c;
+            coord_scale(bp, j, alpha, c);
+            const int q = round_checked<ROUND>(__fmul_rn(alpha, grad_at<GRAD>(g, j)), wv[t], P.Lf, clip_slot, nonf_slot);
+            if (PAY == INTSGD_PAYLOAD_I32) ((int32_t*)out)[j] = q;
+            else ((int8_t*)out)[j] = (int8_t)q;
+        }
+    }
+    counters_flush(s_cnt, st);
+}
+
+// Aggregate + decode + update with block-wise decode factors and per-segment squared step lengths (Algorithm 2:
+// every block is decoded with its own eta / (n alpha_{k,l})).  One unit per thread and iteration for both wire
+// types, so that a warp's 32 units are one chunk of the norm reduction.
+template <int PAY, bool ALIGNED>
+__global__ void __launch_bounds__(512) aggregate_blocks_kernel(const __grid_constant__ VecParams P) {
+    DevState* st = P.st;
+    if (st->status != INTSGD_OK) return;
+    const BlockParams& bp = P.bp;
+    const int n = P.n;
+    const int lane = threadIdx.x & 31;
+    ThreadAcc acc = {0.0, 0, 0u};
+    const int64_t full = P.d >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x - lane); base < full; base += stride) {
+        const int64_t unit = base + lane;
+        int s_lo, s_hi;
+        chunk_segments(bp, base, s_lo, s_hi);
+        double sq[4] = {0.0, 0.0, 0.0, 0.0};
+        int seg[4] = {-1, -1, -1, -1};
+        if (unit < full) {
+            const UnitScale us = unit_scale(bp, unit, s_lo, s_hi);
+            int4 S = make_int4(0, 0, 0, 0);
+#pragma unroll 4
+            for (int i = 0; i < n; ++i) {
+                if (PAY == INTSGD_PAYLOAD_I32) {
+                    const int4 q = load_i4<ALIGNED>((const int32_t*)P.in[i], unit);
+                    S.x += q.x; S.y += q.y; S.z += q.z; S.w += q.w;
+                } else if (ALIGNED) {
+                    add_bytes(S, __ldcs((const uint32_t*)P.in[i] + unit));
+                } else {
+                    const int8_t* p = (const int8_t*)P.in[i] + 4 * unit;
+                    S.x += (int)p[0]; S.y += (int)p[1]; S.z += (int)p[2]; S.w += (int)p[3];
+                }
             }
             const float4 xo = load_f4<ALIGNED>(P.x, unit);
             float4 xn;
@@ -328,16 +544,8 @@ __global__ void __launch_bounds__(512) fused_step_blocks_kernel(const __grid_con
             float alpha, c;
             coord_scale(bp, j, alpha, c);
             int S = 0;
-            for (int i = 0; i < n; ++i) {
-                uint32_t word = 0;
-                if (ROUND != INTSGD_ROUND_NEAREST) {
-                    const uint4 w4 = draw_unit<ROUND>(j >> 2, (uint32_t)i, step, P.keys);
-                    const uint32_t wv[4] = {w4.x, w4.y, w4.z, w4.w};
-                    word = wv[j & 3];
-                }
-                const float y = __fmul_rn(alpha, grad_at<GRAD>(P.in[i], j));
-                S += round_checked<ROUND>(y, word, P.Lf, &s_cnt[i], nonf_slot);
-            }
+            for (int i = 0; i < n; ++i)
+                S += (PAY == INTSGD_PAYLOAD_I32) ? ((const int32_t*)P.in[i])[j] : (int)((const int8_t*)P.in[i])[j];
             double sqj;
             P.x[j] = update_coord_sq(P.x[j], __int2float_rn(S), c, sqj);
             if (P.agg) P.agg[j] = S;
@@ -345,61 +553,7 @@ __global__ void __launch_bounds__(512) fused_step_blocks_kernel(const __grid_con
             bp.tail_sq[j - bp.covered_end] = sqj;
         }
     }
-    counters_flush(s_cnt, st);
     flush_sum_counters(acc, st);
-}
-
-// Exact first step with per-segment squared step lengths (Algorithm 2's Input line: x^1 is the
-// uncompressed mean step; its block norms start the moving averages).
-template <int GRAD, bool ALIGNED>
-__global__ void __launch_bounds__(512) exact_step_blocks_kernel(const __grid_constant__ VecParams P) {
-    const BlockParams& bp = P.bp;
-    const int n = P.n;
-    const float c0 = P.c_exact;
-    const int lane = threadIdx.x & 31;
-    const int64_t full = P.d >> 2;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x - lane); base < full; base += stride) {
-        const int64_t unit = base + lane;
-        const bool active = unit < full;
-        int s_lo, s_hi;
-        chunk_segments(bp, base, s_lo, s_hi);
-        double sq[4] = {0.0, 0.0, 0.0, 0.0};
-        int seg[4] = {-1, -1, -1, -1};
-        if (active) {
-            float4 m = load_grad4<GRAD, ALIGNED>(P.in[0], unit);
-#pragma unroll 4
-            for (int i = 1; i < n; ++i) {
-                const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
-                m.x = __fadd_rn(m.x, gv.x); m.y = __fadd_rn(m.y, gv.y);
-                m.z = __fadd_rn(m.z, gv.z); m.w = __fadd_rn(m.w, gv.w);
-            }
-            const float4 xo = load_f4<ALIGNED>(P.x, unit);
-            float4 xn;
-            xn.x = update_coord_sq(xo.x, m.x, c0, sq[0]);
-            xn.y = update_coord_sq(xo.y, m.y, c0, sq[1]);
-            xn.z = update_coord_sq(xo.z, m.z, c0, sq[2]);
-            xn.w = update_coord_sq(xo.w, m.w, c0, sq[3]);
-            store_f4<ALIGNED>(P.x, unit, xn);
-            if (s_lo == s_hi) {
-                seg[0] = seg[1] = seg[2] = seg[3] = s_lo;
-            } else {
-                const UnitScale us = unit_scale(bp, unit, s_lo, s_hi);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
-            }
-        }
-        chunk_commit(bp, base, s_lo, s_hi, sq, seg);
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        for (int64_t j = full << 2; j < P.d; ++j) {
-            float m = grad_at<GRAD>(P.in[0], j);
-            for (int i = 1; i < n; ++i) m = __fadd_rn(m, grad_at<GRAD>(P.in[i], j));
-            double sqj;
-            P.x[j] = update_coord_sq(P.x[j], m, c0, sqj);
-            bp.tail_sq[j - bp.covered_end] = sqj;
-        }
-    }
 }
 
 }  // namespace intsgd

@@ -48,6 +48,13 @@ struct PhiloxKeys {
     uint32_t k1[10];
 };
 
+// Round-1/round-2 Philox values that depend only on (seed, worker) when the high counter word is
+// zero (d <= 2^34): computed on the host once per context, copied to shared memory by each block.
+// Entry i: x = lo(M1 * i) ^ k0[1];  y = hi(M0 * n0) ^ k1[1] with n0 = hi(M1 * i) ^ k0[0];  z = lo(M0 * n0).
+struct PhiloxWorkerTable {
+    uint4 e[INTSGD_MAX_WORKERS];
+};
+
 // Block-wise scales (Algorithm 2); B == 0 means one scalar alpha (Algorithm 1).  See intsgd_blocks.cuh.
 struct BlockParams {
     const int64_t* offsets;   // device, B + 1 entries, offsets[0] = 0, offsets[B] = d
@@ -88,6 +95,7 @@ struct VecParams {
     int64_t unit_base;
     int32_t window_flags;
     PhiloxKeys keys;
+    PhiloxWorkerTable tab;
     BlockParams bp;
 };
 
@@ -100,6 +108,38 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
                                                const PhiloxKeys& K) {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ K.k1[r];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// Philox4x32-10 for counter (unit, 0, worker, step) with rounds 1-2 folded:
+// per tile and thread: p0 = M0 * unit -> n3 = lo, n2 = hi ^ step ^ k1[0]; p1' = M1 * n2 -> H, m1.
+// per worker: m0 = H ^ e[i].x, m2 = e[i].y ^ n3, m3 = e[i].z; then rounds 3..10.
+struct PhiloxThreadPart {
+    uint32_t n3, H, m1;
+};
+__device__ __forceinline__ PhiloxThreadPart philox_thread_part(uint32_t unit_lo, uint32_t step, const PhiloxKeys& K) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)unit_lo;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ step ^ K.k1[0];
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)n2;
+    PhiloxThreadPart t;
+    t.n3 = (uint32_t)p0;
+    t.H = (uint32_t)(p1 >> 32);
+    t.m1 = (uint32_t)p1;
+    return t;
+}
+__device__ __forceinline__ uint4 philox_finish(const PhiloxThreadPart& t, uint4 e, const PhiloxKeys& K) {
+    uint32_t c0 = t.H ^ e.x, c1 = t.m1, c2 = e.y ^ t.n3, c3 = e.z;
+#pragma unroll
+    for (int r = 2; r < 10; ++r) {
         const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
         const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
         const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
@@ -127,6 +167,32 @@ __device__ __forceinline__ uint4 draw_unit(int64_t unit, uint32_t worker, uint32
         return make_uint4(a & 0xFFFFu, a >> 16, b & 0xFFFFu, b >> 16);
     }
     return philox4x32_10((uint32_t)unit, (uint32_t)((uint64_t)unit >> 32), worker, step, K);
+}
+
+// The same draws with rounds 1-2 folded, for a kernel that keeps a unit across several workers (or a worker
+// across several units): draw_thread_part is the unit's half (2 wide multiplies), `e` the worker's half
+// (PhiloxWorkerTable entry), draw_unit_folded the remaining rounds (16 wide multiplies).  The folding needs a
+// zero high counter word; beyond 2^32 blocks the full ten rounds run.
+template <int ROUND>
+__device__ __forceinline__ uint64_t draw_block_index(int64_t unit) {
+    const uint64_t u = (uint64_t)unit;
+    return (ROUND == INTSGD_ROUND_RANDOM16) ? (((u >> 10) << 9) | (u & 511)) : u;
+}
+template <int ROUND>
+__device__ __forceinline__ PhiloxThreadPart draw_thread_part(int64_t unit, uint32_t step, const PhiloxKeys& K) {
+    return philox_thread_part((uint32_t)draw_block_index<ROUND>(unit), step, K);
+}
+template <int ROUND>
+__device__ __forceinline__ uint4 draw_unit_folded(const PhiloxThreadPart& tp, int64_t unit, uint4 e, uint32_t worker,
+                                                  uint32_t step, const PhiloxKeys& K) {
+    const uint64_t idx = draw_block_index<ROUND>(unit);
+    const uint4 w = (idx >> 32) ? philox4x32_10((uint32_t)idx, (uint32_t)(idx >> 32), worker, step, K) : philox_finish(tp, e, K);
+    if (ROUND == INTSGD_ROUND_RANDOM16) {
+        const bool h = ((uint64_t)unit >> 9) & 1;
+        const uint32_t a = h ? w.z : w.x, b = h ? w.w : w.y;
+        return make_uint4(a & 0xFFFFu, a >> 16, b & 0xFFFFu, b >> 16);
+    }
+    return w;
 }
 
 // The uniform draw is draw_as_float(w) * draw_scale(): the word times 2^-32 truncated to fp32 (the
@@ -205,6 +271,33 @@ __device__ __forceinline__ int4 load_i4(const int32_t* base, int64_t unit) {
     if (ALIGNED) return __ldcs((const int4*)base + unit);
     const int32_t* p = base + 4 * unit;
     return make_int4(__ldcs(p), __ldcs(p + 1), __ldcs(p + 2), __ldcs(p + 3));
+}
+
+// Four payload values of one unit: int32 as one 16-byte store, int8 as the four low bytes packed into one word.
+template <int PAY>
+__device__ __forceinline__ void store_payload4(void* base, int64_t unit, int4 q, bool aligned) {
+    if (PAY == INTSGD_PAYLOAD_I32) {
+        if (aligned) { __stcs((int4*)base + unit, q); return; }
+        int32_t* p = (int32_t*)base + 4 * unit;
+        __stcs(p, q.x); __stcs(p + 1, q.y); __stcs(p + 2, q.z); __stcs(p + 3, q.w);
+    } else {
+        if (aligned) {
+            // low bytes of the four values, in order
+            const uint32_t packed = __byte_perm(__byte_perm(q.x, q.y, 0x0040), __byte_perm(q.z, q.w, 0x0040), 0x5410);
+            __stcs((uint32_t*)base + unit, packed);
+            return;
+        }
+        int8_t* p = (int8_t*)base + 4 * unit;
+        p[0] = (int8_t)q.x; p[1] = (int8_t)q.y; p[2] = (int8_t)q.z; p[3] = (int8_t)q.w;
+    }
+}
+
+// Adds the four signed bytes of one packed int8 unit to the four sums.
+__device__ __forceinline__ void add_bytes(int4& s, uint32_t v) {
+    s.x += (int)(int8_t)(v & 0xFF);
+    s.y += (int)(int8_t)((v >> 8) & 0xFF);
+    s.z += (int)(int8_t)((v >> 16) & 0xFF);
+    s.w += (int)(int8_t)(v >> 24);
 }
 
 // max(|a|, |b|, |c|), NaN if any input is NaN (three-input max of sm_100).

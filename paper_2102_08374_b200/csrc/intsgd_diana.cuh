@@ -54,13 +54,15 @@ __global__ void __launch_bounds__(512) diana_step_kernel(const __grid_constant__
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
         int4 S = make_int4(0, 0, 0, 0);
+        PhiloxThreadPart tp = {0u, 0u, 0u};   // the unit's half of Philox rounds 1-2 serves all n workers
+        if (ROUND != INTSGD_ROUND_NEAREST) tp = draw_thread_part<ROUND>(unit, step, P.keys);
 #pragma unroll 2
         for (int i = 0; i < n; ++i) {
             const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
             float* hl = (float*)P.out[i];
             float4 hv = load_f4<ALIGNED>(hl, unit);
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, (uint32_t)i, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit_folded<ROUND>(tp, unit, P.tab.e[i], (uint32_t)i, step, P.keys);
             S.x += diana_worker_coord<ROUND>(gv.x, hv.x, w.x, f, P.Lf, &s_cnt[i], nonf_slot);
             S.y += diana_worker_coord<ROUND>(gv.y, hv.y, w.y, f, P.Lf, &s_cnt[i], nonf_slot);
             S.z += diana_worker_coord<ROUND>(gv.z, hv.z, w.z, f, P.Lf, &s_cnt[i], nonf_slot);
@@ -152,7 +154,7 @@ __global__ void __launch_bounds__(NC + 32, 1) diana_pipe_kernel(const __grid_con
         s_fault = 0;
         mbar_fence_init();
     }
-    for (int i = threadIdx.x; i < INTSGD_MAX_WORKERS; i += blockDim.x) s_tab[i] = PP.tab.e[i];
+    for (int i = threadIdx.x; i < INTSGD_MAX_WORKERS; i += blockDim.x) s_tab[i] = P.tab.e[i];
     counters_init(s_cnt);   // includes a __syncthreads()
     grid_dependency_wait();
     if (st->status != INTSGD_OK) return;
@@ -161,10 +163,11 @@ __global__ void __launch_bounds__(NC + 32, 1) diana_pipe_kernel(const __grid_con
     const int64_t tiles = PP.tiles;
     ThreadAcc acc = {0.0, 0, 0u};
     bool ok = true;
+    uint32_t it = 0;   // producer thread: stages filled so far
 
     if (threadIdx.x >= NC) {
         if (threadIdx.x == NC) {   // producer
-            uint32_t it = 0, s = 0, phase = 0;
+            uint32_t s = 0, phase = 0;
             for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
                 const int64_t left = PP.units - tile * kTileUnits;
                 const uint32_t units = (uint32_t)(left < kTileUnits ? left : kTileUnits);
@@ -183,14 +186,7 @@ __global__ void __launch_bounds__(NC + 32, 1) diana_pipe_kernel(const __grid_con
                     if (++s == NS) { s = 0; phase ^= 1u; }
                 }
             }
-            if (!ok) {
-                atomicExch(&s_fault, 1);
-                const uint32_t pending = it < NS ? it : NS;
-                for (uint32_t k = 0; k < pending; ++k) {
-                    const uint32_t j = it - 1 - k;
-                    mbar_wait(&full_bar[j % NS], (j / NS) & 1u);
-                }
-            }
+            if (!ok) atomicExch(&s_fault, 1);
         }
     } else {
         const int c = threadIdx.x;
@@ -288,6 +284,9 @@ __global__ void __launch_bounds__(NC + 32, 1) diana_pipe_kernel(const __grid_con
             }
         }
     }
+    __syncthreads();
+    // whichever side's wait gave up: the producer thread lets the copies it has issued land before the block retires
+    if (threadIdx.x == NC && s_fault) drain_issued<NS>(full_bar, it);
     counters_flush(s_cnt, st);   // includes a __syncthreads()
     if (threadIdx.x == 0 && s_fault) atomicExch(&st->fault, 1);
     grid_finalize(acc, st, P.partials, true);

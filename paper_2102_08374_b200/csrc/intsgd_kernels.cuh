@@ -50,24 +50,6 @@ __global__ void scale_kernel(DevState* st, double sqrt_d, double two_n, double n
 // ----------------------------------------------------------------------------------------
 // Encode: payload_i = clip(Int(alpha g_i)).  grid = (blocks, workers).
 // ----------------------------------------------------------------------------------------
-template <int PAY>
-__device__ __forceinline__ void store_payload4(void* base, int64_t unit, int4 q, bool aligned) {
-    if (PAY == INTSGD_PAYLOAD_I32) {
-        if (aligned) { __stcs((int4*)base + unit, q); return; }
-        int32_t* p = (int32_t*)base + 4 * unit;
-        __stcs(p, q.x); __stcs(p + 1, q.y); __stcs(p + 2, q.z); __stcs(p + 3, q.w);
-    } else {
-        if (aligned) {
-            // low bytes of the four values, in order
-            const uint32_t packed = __byte_perm(__byte_perm(q.x, q.y, 0x0040), __byte_perm(q.z, q.w, 0x0040), 0x5410);
-            __stcs((uint32_t*)base + unit, packed);
-            return;
-        }
-        int8_t* p = (int8_t*)base + 4 * unit;
-        p[0] = (int8_t)q.x; p[1] = (int8_t)q.y; p[2] = (int8_t)q.z; p[3] = (int8_t)q.w;
-    }
-}
-
 template <int GRAD, int PAY, bool ALIGNED, int ROUND>
 __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_constant__ VecParams P) {
     __shared__ cnt_t s_cnt[INTSGD_MAX_WORKERS + 1];
@@ -82,6 +64,7 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
     void* out = P.out[slot];
     cnt_t* clip_slot = &s_cnt[worker];
     cnt_t* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
+    const uint4 e = P.tab.e[worker];   // the worker's half of Philox rounds 1-2 (fixed for the whole block)
 
     const int64_t full = P.d >> 2;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -90,7 +73,8 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
         for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
             const float4 gv = load_grad4<GRAD, ALIGNED>(g, unit);
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit, worker, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST)
+                w = draw_unit_folded<ROUND>(draw_thread_part<ROUND>(unit, step, P.keys), unit, e, worker, step, P.keys);
             store_payload4<PAY>(out, unit, round_unit<ROUND>(gv, alpha, w, P.Lf, clip_slot, nonf_slot), ALIGNED);
         }
     } else if (ROUND == INTSGD_ROUND_RANDOM16) {
@@ -108,7 +92,8 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
             if (np < pairs && nu < full) ga = load_grad4<GRAD, ALIGNED>(g, nu);
             if (np < pairs && nu + 512 < full) gb = load_grad4<GRAD, ALIGNED>(g, nu + 512);
             ua = nu;
-            const uint4 w = philox4x32_10((uint32_t)pr, (uint32_t)((uint64_t)pr >> 32), worker, step, P.keys);
+            const uint4 w = ((uint64_t)pr >> 32) ? philox4x32_10((uint32_t)pr, (uint32_t)((uint64_t)pr >> 32), worker, step, P.keys)
+                                                 : philox_finish(philox_thread_part((uint32_t)pr, step, P.keys), e, P.keys);
             const uint4 wa = make_uint4(w.x & 0xFFFFu, w.x >> 16, w.y & 0xFFFFu, w.y >> 16);
             const uint4 wb = make_uint4(w.z & 0xFFFFu, w.z >> 16, w.w & 0xFFFFu, w.w >> 16);
             if (ca_unit < full)
@@ -130,8 +115,8 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
             if (nb < full) gb = load_grad4<GRAD, ALIGNED>(g, nb);
             uint4 wa = make_uint4(0, 0, 0, 0), wb = wa;
             if (ROUND != INTSGD_ROUND_NEAREST) {
-                wa = draw_unit<ROUND>(unit, worker, step, P.keys);
-                wb = draw_unit<ROUND>(ub, worker, step, P.keys);
+                wa = draw_unit_folded<ROUND>(draw_thread_part<ROUND>(unit, step, P.keys), unit, e, worker, step, P.keys);
+                wb = draw_unit_folded<ROUND>(draw_thread_part<ROUND>(ub, step, P.keys), ub, e, worker, step, P.keys);
             }
             store_payload4<PAY>(out, unit, round_unit<ROUND>(ca, alpha, wa, P.Lf, clip_slot, nonf_slot), ALIGNED);
             if (ub < full) store_payload4<PAY>(out, ub, round_unit<ROUND>(cb, alpha, wb, P.Lf, clip_slot, nonf_slot), ALIGNED);
@@ -158,13 +143,6 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
 // int32 payloads: one unit (4 coordinates) per thread iteration.
 // int8 payloads : four units (16 coordinates, one 16-byte load per worker) per iteration.
 // ----------------------------------------------------------------------------------------
-__device__ __forceinline__ void add_bytes(int4& s, uint32_t v) {
-    s.x += (int)(int8_t)(v & 0xFF);
-    s.y += (int)(int8_t)((v >> 8) & 0xFF);
-    s.z += (int)(int8_t)((v >> 16) & 0xFF);
-    s.w += (int)(int8_t)(v >> 24);
-}
-
 template <bool ALIGNED>
 __device__ __forceinline__ void apply_unit(const VecParams& P, int64_t unit, int4 S, float c, ThreadAcc& acc) {
     const float4 xo = load_f4<ALIGNED>(P.x, unit);
@@ -265,11 +243,15 @@ __global__ void __launch_bounds__(kMaxThreads) fused_step_kernel(const __grid_co
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t unit = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; unit < full; unit += stride) {
         int4 S = make_int4(0, 0, 0, 0);
+        // the unit's half of Philox rounds 1-2 serves all n workers
+        PhiloxThreadPart tp = {0u, 0u, 0u};
+        if (ROUND != INTSGD_ROUND_NEAREST) tp = draw_thread_part<ROUND>(unit + P.unit_base, step, P.keys);
 #pragma unroll 4
         for (int i = 0; i < n; ++i) {
             const float4 gv = load_grad4<GRAD, ALIGNED>(P.in[i], unit);
             uint4 w = make_uint4(0, 0, 0, 0);
-            if (ROUND != INTSGD_ROUND_NEAREST) w = draw_unit<ROUND>(unit + P.unit_base, (uint32_t)i, step, P.keys);
+            if (ROUND != INTSGD_ROUND_NEAREST)
+                w = draw_unit_folded<ROUND>(tp, unit + P.unit_base, P.tab.e[i], (uint32_t)i, step, P.keys);
             const int4 q = round_unit<ROUND>(gv, alpha, w, P.Lf, &s_cnt[i], nonf_slot);
             S.x += q.x; S.y += q.y; S.z += q.z; S.w += q.w;
         }

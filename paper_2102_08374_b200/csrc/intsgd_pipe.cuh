@@ -9,7 +9,8 @@
 // conflict-free 16-byte (8-byte) accesses and the Philox counters of a thread are fixed for a whole tile.
 //
 // Requirements checked by the host: every pointer 16-byte aligned, d <= 2^34.  Everything else
-// (unaligned pointers, larger d) runs in fused_step_kernel.
+// (unaligned pointers, larger d) runs in fused_step_kernel.  A launch may cover a window of the vector: `unit`
+// indexes the launch's pointers, `unit + unit_base` the whole vector (random stream, partition tables, chunk partials).
 #pragma once
 
 #include "intsgd_blocks.cuh"
@@ -59,6 +60,18 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
                      smem_addr(dst_smem)),
                  "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
                  : "memory");
+}
+
+// Failure path of the pipelined kernels: waits (each wait bounded) until the last min(issued, NS) stages the
+// producer has filled have landed, so that no bulk copy is still in flight into the shared memory of a block
+// that is about to retire.  Stage j (0-based) completes phase (j / NS) & 1 of barrier j % NS.
+template <int NS>
+__device__ __forceinline__ void drain_issued(uint64_t* full_bar, uint32_t issued) {
+    const uint32_t pending = issued < (uint32_t)NS ? issued : (uint32_t)NS;
+    for (uint32_t k = 0; k < pending; ++k) {
+        const uint32_t j = issued - 1 - k;
+        mbar_wait(&full_bar[j % NS], (j / NS) & 1u);
+    }
 }
 
 // ---- per-unit arithmetic ------------------------------------------------------------------------
@@ -124,52 +137,12 @@ __device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float4 
     return make_int4(S[0], S[1], S[2], S[3]);
 }
 
-// Round-1/round-2 Philox values that depend only on (seed, worker) when the high counter word is
-// zero (d <= 2^34): computed on the host once per context, copied to shared memory by each block.
-// Entry i: x = lo(M1 * i) ^ k0[1];  y = hi(M0 * n0) ^ k1[1] with n0 = hi(M1 * i) ^ k0[0];  z = lo(M0 * n0).
-struct PhiloxWorkerTable {
-    uint4 e[INTSGD_MAX_WORKERS];
-};
-
 struct PipeParams {
     VecParams v;
-    PhiloxWorkerTable tab;
     float fast_limit;   // T: fast path handles |alpha g| <= T
     int64_t units;      // units covered by the pipeline (the rest is the scalar tail)
     int64_t tiles;
 };
-
-// Philox4x32-10 for counter (unit, 0, worker, step) with rounds 1-2 folded:
-// per tile and thread: p0 = M0 * unit -> n3 = lo, n2 = hi ^ step ^ k1[0]; p1' = M1 * n2 -> H, m1.
-// per worker: m0 = H ^ e[i].x, m2 = e[i].y ^ n3, m3 = e[i].z; then rounds 3..10.
-struct PhiloxThreadPart {
-    uint32_t n3, H, m1;
-};
-__device__ __forceinline__ PhiloxThreadPart philox_thread_part(uint32_t unit_lo, uint32_t step, const PhiloxKeys& K) {
-    const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)unit_lo;
-    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ step ^ K.k1[0];
-    const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)n2;
-    PhiloxThreadPart t;
-    t.n3 = (uint32_t)p0;
-    t.H = (uint32_t)(p1 >> 32);
-    t.m1 = (uint32_t)p1;
-    return t;
-}
-__device__ __forceinline__ uint4 philox_finish(const PhiloxThreadPart& t, uint4 e, const PhiloxKeys& K) {
-    uint32_t c0 = t.H ^ e.x, c1 = t.m1, c2 = e.y ^ t.n3, c3 = e.z;
-#pragma unroll
-    for (int r = 2; r < 10; ++r) {
-        const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
-        const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
-        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
-        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ K.k1[r];
-        c1 = (uint32_t)p1;
-        c3 = (uint32_t)p0;
-        c0 = n0;
-        c2 = n2;
-    }
-    return make_uint4(c0, c1, c2, c3);
-}
 
 // 16-bit draws: pair index of a unit, and the four draws of its half of the pair's Philox block.
 __device__ __forceinline__ uint32_t pair_index(uint32_t unit_lo) { return ((unit_lo >> 10) << 9) | (unit_lo & 511u); }
@@ -228,7 +201,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         s_fault = 0;
         mbar_fence_init();
     }
-    for (int i = threadIdx.x; i < INTSGD_MAX_WORKERS; i += blockDim.x) s_tab[i] = PP.tab.e[i];
+    for (int i = threadIdx.x; i < INTSGD_MAX_WORKERS; i += blockDim.x) s_tab[i] = P.tab.e[i];
     counters_init(s_cnt);   // includes a __syncthreads()
     // Everything above needs only the kernel's arguments.  When the launch was allowed to start before
     // the step's scale kernel has finished, wait here for that kernel's writes (a no-op otherwise).
@@ -239,11 +212,12 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
     const int64_t tiles = PP.tiles;
     ThreadAcc acc = {0.0, 0, 0u};
     bool ok = true;
+    uint32_t it = 0;   // producer thread: stages filled so far
 
     if (threadIdx.x >= NC) {
         // ------------------------------- producer ---------------------------------------------
         if (threadIdx.x == NC) {
-            uint32_t it = 0, s = 0, phase = 0;   // it: stages filled so far; s = it % NS; phase = (it / NS) & 1
+            uint32_t s = 0, phase = 0;   // s = it % NS; phase = (it / NS) & 1
             for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
                 const int64_t left = PP.units - tile * kTileUnits;
                 const uint32_t bytes = (uint32_t)(left < kTileUnits ? left : kTileUnits) * kUnitBytes;
@@ -259,15 +233,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                     if (++s == NS) { s = 0; phase ^= 1u; }
                 }
             }
-            if (!ok) {
-                // a wait gave up: let every copy still in flight land before this CTA can exit
-                atomicExch(&s_fault, 1);
-                const uint32_t pending = it < NS ? it : NS;
-                for (uint32_t k = 0; k < pending; ++k) {
-                    const uint32_t j = it - 1 - k;
-                    mbar_wait(&full_bar[j % NS], (j / NS) & 1u);
-                }
-            }
+            if (!ok) atomicExch(&s_fault, 1);
         }
     } else {
         // ------------------------------- consumers --------------------------------------------
@@ -289,7 +255,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
             pre_a[k] = pre_c[k] = 0.0f;
             if (BLOCKS) {
                 const int64_t chunk0 = (int64_t)blockIdx.x * kTileUnits + c + (int64_t)k * NC - lane;
-                if (chunk0 < PP.units) ent[k] = chunk_entry(bp, chunk0);
+                if (chunk0 < PP.units) ent[k] = chunk_entry(bp, chunk0 + P.unit_base);
                 pre_a[k] = __ldg(&bp.alpha[ent[k] & 0x7FFFFFFF]);
                 pre_c[k] = __ldg(&bp.c[ent[k] & 0x7FFFFFFF]);
             }
@@ -324,20 +290,20 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 c_uni[k] = 0.0f;
                 if (BLOCKS) {
                     // the warp's 32 units form one chunk; chunks past the covered range are never committed
-                    if (unit - lane < PP.units) chunk_segments_from(bp, ent[k], unit - lane, s_lo[k], s_hi[k]);
+                    if (unit - lane < PP.units) chunk_segments_from(bp, ent[k], unit - lane + P.unit_base, s_lo[k], s_hi[k]);
                     if (active[k]) {
                         if (s_lo[k] == s_hi[k]) {   // the chunk lies in one segment: scale and decode factor are at hand
                             a01[k] = make_float2(pre_a[k], pre_a[k]);
                             a23[k] = a01[k];
                             c_uni[k] = pre_c[k];
                         } else {
-                            const UnitScale us = unit_scale(bp, unit, s_lo[k], s_hi[k]);
+                            const UnitScale us = unit_scale(bp, unit + P.unit_base, s_lo[k], s_hi[k]);
                             a01[k] = us.a01;
                             a23[k] = us.a23;
                         }
                     }
                     const int64_t next_chunk0 = unit - lane + (int64_t)gridDim.x * kTileUnits;
-                    ent_next[k] = (next_chunk0 < PP.units) ? chunk_entry(bp, next_chunk0) : 0;
+                    ent_next[k] = (next_chunk0 < PP.units) ? chunk_entry(bp, next_chunk0 + P.unit_base) : 0;
                 }
             }
             for (int g0 = 0; g0 < n; g0 += G) {
@@ -395,7 +361,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                         double sq[4] = {0.0, 0.0, 0.0, 0.0};
                         int seg[4] = {-1, -1, -1, -1};
                         if (active[k]) {
-                            const UnitScale us = unit_scale(bp, unit, s_lo[k], s_hi[k]);
+                            const UnitScale us = unit_scale(bp, unit + P.unit_base, s_lo[k], s_hi[k]);
                             int4 S;
                             if (ua[k].m <= PP.fast_limit)
                                 S = make_int4(__float2int_rn(ua[k].F01.x), __float2int_rn(ua[k].F01.y),
@@ -414,7 +380,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
 #pragma unroll
                             for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
                         }
-                        chunk_commit(bp, unit - lane, s_lo[k], s_hi[k], sq, seg);
+                        chunk_commit(bp, unit - lane + P.unit_base, s_lo[k], s_hi[k], sq, seg);
                         continue;
                     }
                 } else if (!active[k]) {
@@ -458,7 +424,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 }
                 if (BLOCKS) {   // all 32 lanes of the warp: one partial per chunk, fixed order
                     const double t = warp_tree(unit_sq);
-                    if (lane == 0) __stcg(&bp.chunk_sum[(unit - lane) >> 5], t);
+                    if (lane == 0) __stcg(&bp.chunk_sum[(unit - lane + P.unit_base) >> 5], t);
                 }
             }
 #pragma unroll
@@ -479,7 +445,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
             const int64_t j0 = PP.units << 2;
             for (int64_t j = j0; j < P.d; ++j) {
                 float aj = alpha, cj = cdec;
-                if (BLOCKS) coord_scale(bp, j, aj, cj);
+                if (BLOCKS) coord_scale(bp, j + (P.unit_base << 2), aj, cj);
                 int S = 0;
                 for (int i = 0; i < n; ++i) {
                     uint32_t word = 0;
@@ -496,17 +462,39 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                     P.x[j] = update_coord_sq(P.x[j], __int2float_rn(S), cj, sqj);
                     if (P.agg) P.agg[j] = S;
                     note_sum(S, P.agg_limit, acc);
-                    bp.tail_sq[j - bp.covered_end] = sqj;
+                    bp.tail_sq[j + (P.unit_base << 2) - bp.covered_end] = sqj;
                 } else {
                     apply_coord(P, j, S, cdec, acc);
                 }
             }
         }
     }
+    __syncthreads();
+    // A wait gave up somewhere in this block (the producer's or a consumer's): before the block can retire,
+    // the producer thread lets every copy it has issued land, whichever side noticed.
+    if (threadIdx.x == NC && s_fault) drain_issued<NS>(full_bar, it);
     counters_flush(s_cnt, st);   // includes a __syncthreads()
     if (threadIdx.x == 0 && s_fault) atomicExch(&st->fault, 1);
     if (BLOCKS) flush_sum_counters(acc, st);   // the per-segment norms are finished by block_norm_kernel
     else grid_finalize(acc, st, P.partials, true, P.window_flags);
+}
+
+// Diagnostic: the rate at which an SM gets through rounds 3-10 of Philox4x32-10 when it does nothing else
+// (register-only: no loads, no rounding, no stores).  Every thread runs two independent chains, as a consumer of
+// the pipelined kernels does with its two units, each block's output seeding the next one's input.  The measured
+// rate of 32x32->64-bit products is the ceiling of the random-rounding kernels' arithmetic.
+__global__ void __launch_bounds__(512) philox_rate_kernel(PhiloxKeys keys, uint32_t blocks_per_chain, uint32_t* sink) {
+    PhiloxThreadPart a, b;
+    a.n3 = threadIdx.x; a.H = blockIdx.x; a.m1 = 0x9E3779B9u;
+    b.n3 = ~threadIdx.x; b.H = blockIdx.x * 7919u; b.m1 = 0xBB67AE85u;
+    uint4 ea = make_uint4(1u, 2u, 3u, 0u), eb = make_uint4(4u, 5u, 6u, 0u);
+    for (uint32_t i = 0; i < blocks_per_chain; ++i) {
+        const uint4 ra = philox_finish(a, ea, keys), rb = philox_finish(b, eb, keys);
+        a.H = ra.x; a.m1 = ra.y; a.n3 = ra.z; ea.z = ra.w;
+        b.H = rb.x; b.m1 = rb.y; b.n3 = rb.z; eb.z = rb.w;
+    }
+    // keeps the chains alive; the condition is all but impossible, so nothing is written in practice
+    if ((a.H ^ b.H ^ a.n3 ^ b.n3) == 0x5EEDu && (a.m1 ^ b.m1 ^ ea.z ^ eb.z) == 0xFACEu) *sink = a.H;
 }
 
 // Diagnostic: the bounded wait on a barrier that nothing completes.  One thread polls `polls` times, then

@@ -48,22 +48,39 @@ def test_multi_step_lockstep(which, grad_dtype, payload_dtype, rounding):
         ls.close()
 
 
-def test_two_kernel_payloads_match_the_oracle():
-    n, d, eta, seed = 4, (1 << 17) + 1, 0.2, 1234
+@pytest.mark.parametrize("d", [(1 << 17) + 1, 4 * 2049 + 3, 2 * 4096, 9, 8])
+@pytest.mark.parametrize("grad_dtype,payload_dtype,rounding", [
+    (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM), (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM),
+    (pkg.GRAD_BF16, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM), (pkg.GRAD_BF16, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM16),
+    (pkg.GRAD_F32, pkg.PAYLOAD_I8, pkg.ROUND_RANDOM16), (pkg.GRAD_F32, pkg.PAYLOAD_I32, pkg.ROUND_RANDOM_COMPARE),
+    (pkg.GRAD_BF16, pkg.PAYLOAD_I8, pkg.ROUND_NEAREST)])
+def test_two_kernel_payloads_match_the_oracle(d, grad_dtype, payload_dtype, rounding):
+    """The payloads that the two-kernel step leaves in the caller's buffers are the oracle's encode of every worker
+    (all workers in one launch of the pipelined encode kernel: whole tiles, a partial tile, the bf16 pair rule and
+    the element-wise tail), with a few clipped and non-finite values planted."""
+    n, eta, seed = 5, 0.2, 1234
     rng = np.random.default_rng(3)
-    for payload_dtype in (pkg.PAYLOAD_I32, pkg.PAYLOAD_I8):
-        ls = LockStep(n, d, payload_dtype=payload_dtype, seed=seed, x0=rng.normal(0, 1, d).astype(np.float32))
-        try:
-            g = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
-            ls.exact(g, eta)
-            g = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
+
+    def grads():
+        out = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
+        out[1][rng.integers(0, d, 4)] = [np.inf, -1e30, np.nan, 7.0]
+        out[3][d - 1] = -np.inf
+        return [synth.to_bf16_bits(g) for g in out] if grad_dtype == pkg.GRAD_BF16 else out
+
+    ls = LockStep(n, d, grad_dtype=grad_dtype, payload_dtype=payload_dtype, rounding=rounding, seed=seed,
+                  x0=rng.normal(0, 1, d).astype(np.float32))
+    try:
+        clean = [rng.normal(0, 1e-2, d).astype(np.float32) for _ in range(n)]
+        ls.exact([synth.to_bf16_bits(g) for g in clean] if grad_dtype == pkg.GRAD_BF16 else clean, eta)
+        for k in (1, 2):
+            g = grads()
             st, ref = ls.step(g, eta, mode=pkg.MODE_TWO_KERNEL)
             for i in range(n):
-                want, _, _ = oracle.encode(g[i], np.float32(st["alpha"]), worker=i, step=1, seed=seed, n=n,
-                                           payload_dtype=payload_dtype)
-                assert np.array_equal(ls.last_payloads[i], want)
-        finally:
-            ls.close()
+                want, _, _ = oracle.encode(g[i], np.float32(st["alpha"]), worker=i, step=k, seed=seed, n=n,
+                                           payload_dtype=payload_dtype, rounding=rounding)
+                assert np.array_equal(ls.last_payloads[i], want), (k, i)
+    finally:
+        ls.close()
 
 
 @pytest.mark.parametrize("which", [FUSED_PIPELINED, FUSED_DIRECT, TWO_KERNEL])
