@@ -214,18 +214,6 @@ int intsgd_set_blocks(intsgd_ctx* ctx, int32_t num_blocks, const int64_t* offset
 int intsgd_get_block_state(intsgd_ctx* ctx, double* r, double* dx2, float* alpha, float* c);
 int intsgd_set_block_state(intsgd_ctx* ctx, const double* r, const double* dx2);
 
-/* Tuning knob: threads per block (multiple of 32, <= 512) and resident blocks per SM used to
- * size the grids of the vector kernels.  0 keeps the built-in value.  Results do not depend on
- * it except the summation order of dx2. */
-int intsgd_set_launch(intsgd_ctx* ctx, int32_t threads_per_block, int32_t blocks_per_sm);
-
-/* Which kernel runs INTSGD_MODE_FUSED: 0 = automatic (the pipelined kernel -- bulk asynchronous copies
- * into a shared-memory ring -- when every pointer is 16-byte aligned and d <= 2^34, else the direct
- * kernel), 1 = always the direct kernel, 2 = same as 0, 3 and 4 = the pipelined kernel with other
- * tile shapes (kept for tuning).  All give identical x, aggregate and counters; dx2 differs only
- * by summation order. */
-int intsgd_set_fused_path(intsgd_ctx* ctx, int32_t path);
-
 /* Diagnostic of the failure path.  Every wait inside the pipelined kernels is bounded; when one gives up the
  * kernel sets a sticky flag, lets its copies in flight land and returns, and intsgd_get_stats reports
  * INTSGD_ERR_TIMEOUT until intsgd_set_state clears the flag.  This call enqueues a one-thread kernel that runs

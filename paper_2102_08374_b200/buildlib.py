@@ -10,7 +10,7 @@ ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libintsgd.so"
 SOURCES = [CSRC / "intsgd.cu", CSRC / "intsgd_noalloc.cu"]
-HEADERS = [CSRC / "intsgd_device.cuh", CSRC / "intsgd_kernels.cuh", CSRC / "intsgd_pipe.cuh", CSRC / "intsgd_blocks.cuh", CSRC / "intsgd_diana.cuh", CSRC / "intsgd_encode_pipe.cuh", ROOT / "include" / "intsgd.h"]
+HEADERS = [CSRC / "intsgd_device.cuh", CSRC / "intsgd_kernels.cuh", CSRC / "intsgd_pipe.cuh", CSRC / "intsgd_blocks.cuh", CSRC / "intsgd_diana.cuh", CSRC / "intsgd_encode_pipe.cuh", ROOT / "include" / "intsgd.h", ROOT / "include" / "intsgd_tuning.h"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

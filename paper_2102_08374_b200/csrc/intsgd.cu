@@ -8,6 +8,7 @@
 #include <new>
 #include <vector>
 
+#include "intsgd_tuning.h"
 #include "intsgd_diana.cuh"
 #include "intsgd_encode_pipe.cuh"
 #include "intsgd_kernels.cuh"
@@ -21,8 +22,7 @@ struct intsgd_ctx {
     float Lf;             // largest fp32 <= L
     PhiloxKeys keys;
     PhiloxWorkerTable tab;
-    int fused_path;       // 0 = automatic, 1 = direct (register) kernel, 2.. = pipelined kernel
-    int pipe_variant;     // index into kPipeShapes
+    int fused_path;       // 0 / 2 = automatic (pipelined kernels when the pointers allow it), 1 = direct kernels
     DevState* d_state;
     double* d_partials;
     int max_grid;
@@ -300,20 +300,15 @@ void launch_fused_r(const intsgd_ctx* ctx, const VecParams& P, int grid, cudaStr
         fused_step_kernel<GRAD, ALIGNED, INTSGD_ROUND_RANDOM><<<grid, ctx->threads, 0, s>>>(P);
 }
 
-// Pipelined kernel shapes: NC consumer threads (+ one producer warp), UPT units per thread and
-// tile, G worker tiles per stage, NS stages; one block per SM, <= 192 KiB of shared memory.
+// Pipelined kernel shape: NC consumer threads (+ one producer warp), UPT units per thread and tile, G worker
+// tiles per stage, NS stages; one block per SM, 192 KiB of shared memory.  512 x 2 units with 3 stages of 4 fp32
+// (8 bf16) worker tiles is the fastest of the shapes timed on B200 (one or four units per thread, 256 to 992
+// consumers, two smaller blocks per SM: all slower).
 struct PipeShape { int nc, upt, g, ns; };
-constexpr PipeShape kPipeShapes[] = {
-    {512, 2, 4, 3},   // variant 0 (path 0 and 2): the default, fastest of the shapes tried on B200
-    {512, 1, 4, 6},   // variant 1 (path 3): one unit per thread, deeper ring
-    {256, 4, 4, 3},   // variant 2 (path 4): fewer, fatter threads
-};
-constexpr int kNumPipeShapes = sizeof(kPipeShapes) / sizeof(kPipeShapes[0]);
-
-template <int GRAD, int ROUND, bool BLOCKS, int V>
+template <int GRAD, int ROUND, bool BLOCKS>
 cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
-    // bf16 tiles are half as large: the default shape stages 8 worker tiles at a time (fewer barrier rounds)
-    constexpr PipeShape S = (GRAD == INTSGD_GRAD_BF16 && V == 0) ? PipeShape{512, 2, 8, 3} : kPipeShapes[V];
+    // bf16 tiles are half as large: a stage holds 8 worker tiles (fewer barrier rounds)
+    constexpr PipeShape S = (GRAD == INTSGD_GRAD_BF16) ? PipeShape{512, 2, 8, 3} : PipeShape{512, 2, 4, 3};
     auto kernel = fused_pipe_kernel<GRAD, ROUND, BLOCKS, S.nc, S.upt, S.g, S.ns>;
     const int unit_bytes = (GRAD == INTSGD_GRAD_F32) ? 16 : 8;
     const int smem = S.ns * S.g * S.nc * S.upt * unit_bytes;
@@ -344,12 +339,7 @@ cudaError_t launch_pipe_v(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s)
 }
 template <int GRAD, int ROUND>
 cudaError_t launch_pipe_t(const intsgd_ctx* ctx, PipeParams& PP, cudaStream_t s) {
-    if (ctx->bs.B > 0) return launch_pipe_v<GRAD, ROUND, true, 0>(ctx, PP, s);   // block-wise: default shape only
-    switch (ctx->pipe_variant) {
-        case 1: return launch_pipe_v<GRAD, ROUND, false, 1>(ctx, PP, s);
-        case 2: return launch_pipe_v<GRAD, ROUND, false, 2>(ctx, PP, s);
-        default: return launch_pipe_v<GRAD, ROUND, false, 0>(ctx, PP, s);
-    }
+    return ctx->bs.B > 0 ? launch_pipe_v<GRAD, ROUND, true>(ctx, PP, s) : launch_pipe_v<GRAD, ROUND, false>(ctx, PP, s);
 }
 // `d` is the length of the launch (a window of the vector, or all of it).
 bool pipe_eligible(const intsgd_ctx* ctx, bool aligned, int64_t d) {
@@ -1276,10 +1266,9 @@ int intsgd_set_launch(intsgd_ctx* ctx, int32_t threads_per_block, int32_t blocks
 
 int intsgd_set_fused_path(intsgd_ctx* ctx, int32_t path) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
-    if (path < 0 || path >= 2 + kNumPipeShapes)
-        return fail(ctx, INTSGD_ERR_INVALID_ARG, "path must be 0 (auto), 1 (direct) or 2.. (pipelined shapes)");
+    if (path < 0 || path > 2)
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "path must be 0 (automatic), 1 (direct kernels) or 2 (same as 0)");
     ctx->fused_path = path;
-    ctx->pipe_variant = path >= 2 ? path - 2 : 0;
     return INTSGD_OK;
 }
 

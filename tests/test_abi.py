@@ -11,9 +11,13 @@ ROOT = Path(__file__).resolve().parent.parent
 
 
 def _declared_symbols():
-    text = (ROOT / "include" / "intsgd.h").read_text()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(intsgd_[a-z_0-9]+)\s*\(", text)))
+    """Every entry point declared in the public header and in the header of the test / tuning knobs."""
+    names = set()
+    for header in ("intsgd.h", "intsgd_tuning.h"):
+        text = (ROOT / "include" / header).read_text()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(intsgd_[a-z_0-9]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_header_and_binding_list_the_same_entry_points():

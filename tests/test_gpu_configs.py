@@ -21,6 +21,12 @@ def _dx2_fp64(x_after, x_before):
     return float(((x_after - x_before).double() ** 2).sum().item())
 
 
+def _clipped(g, alpha_t, limit):
+    """Coordinates of one worker whose scaled value leaves the clip range: the counter's definition, evaluated
+    with one separately rounded fp32 multiply on the device."""
+    return int((~((g * alpha_t).abs() <= limit)).sum().item())
+
+
 class ScalarChain:
     """The oracle's scalar recursion (r_k, alpha_k, c_k) driven by the measured step lengths."""
 
@@ -86,6 +92,42 @@ def test_config2_logistic_regression_500_steps():
         ls.close()
 
 
+def test_heterogeneous_workers_drive_the_integers_past_2_23_and_into_the_clip():
+    """Appendix A.2 / C.5 of the paper: on heterogeneous data the local gradients do not vanish at the optimum, so
+    as the iterates converge alpha_k grows and the transmitted integers grow with it.  A small, strongly
+    heterogeneous logistic regression (64 workers of 8 samples) is driven, in lock step with the oracle on the
+    whole vector every step, through three regimes: values beyond the pipelined kernel's float-accumulation range
+    (redone exactly), |alpha g| >= 2^23 (no fractional bits: Int is deterministic), and the int32 clip limit
+    floor((2^31 - 1) / n) (counted, after which the large step makes alpha collapse and regrow)."""
+    n, m, d, eta, steps, seed = 64, 8, 256, 0.5, 300, 2
+    prob = synth.LogisticProblem(n=n, m=m, d=d, lam=0.1, device=dev())
+    limit = oracle.limit_as_float(oracle.default_clip_limit(n, pkg.PAYLOAD_I32))
+    paths = [(pkg.MODE_FUSED, 0), (pkg.MODE_TWO_KERNEL, 0), (pkg.MODE_FUSED, 1)]
+    ls = LockStep(n, d, seed=seed, beta=0.5, x0=np.zeros(d, dtype=np.float32))
+    try:
+        beyond_fast = beyond_23 = clipped_steps = 0
+        max_int = 0
+        for k in range(steps):
+            g_dev = prob.gradients(ls.x_dev)
+            grads = [to_host(g) for g in g_dev]
+            if k == 0:
+                ls.exact(grads, eta)
+                continue
+            mode, path = paths[k % 3]
+            ls.lib.intsgd_set_fused_path(path)
+            st, ref = ls.step(grads, eta, mode=mode, g_dev=g_dev)
+            ymax = st["alpha"] * max(float(np.abs(g).max()) for g in grads)
+            beyond_fast += ymax > (1 << 24) / n
+            beyond_23 += ymax >= 2.0 ** 23
+            clipped_steps += sum(st["clip_count"]) > 0
+            max_int = max(max_int, st["max_abs_agg"])
+            assert ymax <= limit or sum(st["clip_count"]) > 0
+        assert beyond_fast > 20 and beyond_23 > 3 and clipped_steps >= 1
+        assert max_int > 1 << 20        # the clipped step's aggregate is no longer a sum of cancelling integers
+    finally:
+        ls.close()
+
+
 def test_config3_resnet18_shaped_200_steps():
     n, d, eta, steps, seed, pool = 16, synth.RESNET18_D, 0.1, 200, 3, 4
     assert d % 4 == 2
@@ -96,7 +138,7 @@ def test_config3_resnet18_shaped_200_steps():
     chain = ScalarChain(n, d)
     # windows: start, the ragged end, one that crosses several small (batch-norm) segments
     windows = [(0, 1 << 15), (d - 30_001, d), (1728 + 64, 1728 + 64 + 40_000), (5_000_001, 5_000_001 + (1 << 15))]
-    full_steps = {1, 2}
+    full_steps = {1, 2, 150}      # the whole vector, counters included: two early steps and a late one
     sampled = {1, 2, 3, 50, 101, 150, 199}
     with pkg.IntSGD(n, d, seed=seed) as lib:
         dx2_prev = None
@@ -121,6 +163,7 @@ def test_config3_resnet18_shaped_200_steps():
                 assert np.array_equal(to_host(x).view(np.uint32), x_ref.view(np.uint32))
                 assert rel_close(st["dx2"], ref["dx2"])
                 assert st["clip_count"] == ref["clip_count"] and st["max_abs_agg"] == ref["max_abs_agg"]
+                assert st["nonfinite"] == ref["nonfinite"] and st["agg_overflow"] == ref["agg_overflow"]
             elif k in sampled:
                 for (j0, j1) in windows:
                     check_window(st, g, x_before, x, agg, j0, j1, step=k, seed=seed, n=n)
@@ -157,7 +200,7 @@ def test_config4_lstm_shaped_bf16_int8_200_steps():
                 x_ref = to_host(x_before)
                 ref_dx2 = oracle.exact_step([to_host(t) for t in g], x_ref, eta)
                 assert np.array_equal(to_host(x), x_ref) and rel_close(st["dx2"], ref_dx2)
-            elif k == 1:   # the whole vector once, counters included
+            elif k in (1, 101):   # the whole vector, counters included: at the start and right after eta drops (alpha jumps)
                 x_ref = to_host(x_before)
                 ref = oracle.step_window([to_host(t) for t in g], x_ref, np.float32(st["alpha"]), np.float32(st["c"]),
                                          step=k, seed=seed, payload_dtype=pkg.PAYLOAD_I8)
@@ -215,12 +258,20 @@ def test_config5_bucket_sweep(log2d, n):
                         if k == 1:
                             chain.r = 0.0
                             chain.advance(eta, dx2_prev, st)
+                        limit = oracle.limit_as_float(oracle.default_clip_limit(n, payload_dtype))
+                        alpha_t = torch.tensor(st["alpha"], dtype=torch.float32, device=dev())
                         for (j0, j1) in windows:
-                            check_window(st, grads, x_before, x, agg, j0, j1, step=k, seed=seed, n=n,
-                                         payload_dtype=payload_dtype)
+                            ref = check_window(st, grads, x_before, x, agg, j0, j1, step=k, seed=seed, n=n,
+                                               payload_dtype=payload_dtype)
+                            # the oracle's counters on the window against the counter's definition, !(|fl32(alpha g)| <= Lf)
+                            assert ref["clip_count"] == [_clipped(g[j0:j1], alpha_t, limit) for g in grads]
+                            assert ref["max_abs_agg"] == int(agg[j0:j1].abs().max().item())
                         assert rel_close(st["dx2"], _dx2_fp64(x, x_before))
                         assert st["max_abs_agg"] == int(agg.abs().max().item())
-                        assert sum(st["clip_count"]) == 0 and st["nonfinite"] == 0
+                        # the library's counters on the whole vector against the same definition
+                        assert st["clip_count"] == [_clipped(g, alpha_t, limit) for g in grads]
+                        assert st["nonfinite"] == 0
+                        assert st["agg_overflow"] == (int((agg.abs() > 127).sum().item()) if payload_dtype == pkg.PAYLOAD_I8 else 0)
                     if k == 0:
                         dx2_prev = st["dx2"]
                 assert lib.intsgd_get_stats()["step"] == steps

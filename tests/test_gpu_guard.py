@@ -68,7 +68,7 @@ SIZES = [1, 3, 7, 12, 1023, (1 << 16) + 2, 8200 + 5, 2 * 1024 * 4 + 4 + 3]   # i
 @pytest.mark.parametrize("d", SIZES)
 @pytest.mark.parametrize("bf16", [False, True])
 @pytest.mark.parametrize("shift", [0, 1])
-@pytest.mark.parametrize("path", [0, 1, 3, 4])
+@pytest.mark.parametrize("path", [0, 1])
 def test_fused_and_exact_steps_stay_inside_x_and_agg(d, bf16, shift, path):
     n = 3
     g = grads_for(n, d, bf16)
