@@ -416,7 +416,6 @@ void fill_block_params(const intsgd_ctx* ctx, VecParams& P, int64_t covered_end)
     P.bp.c = ctx->bs.c;
     P.bp.chunk_sum = ctx->bs.chunk_sum;
     P.bp.chunk_seg = ctx->bs.chunk_seg;
-    P.bp.tile_seg = ctx->bs.tile_seg;
     P.bp.edge_sum = ctx->bs.edge_sum;
     P.bp.tail_sq = ctx->bs.tail_sq;
     P.bp.covered_end = covered_end;
@@ -1184,9 +1183,8 @@ int intsgd_set_blocks(intsgd_ctx* ctx, int32_t num_blocks, const int64_t* offset
     CUDA_TRY(ctx, cudaMalloc(&ctx->d_offsets, (B + 1) * sizeof(int64_t)));
     cudaError_t e = cudaMalloc(&base, bytes);
     double* chunk = nullptr;
-    // chunk partials (double) followed by the chunk -> segment table and the tile -> segment table (int32)
-    const size_t tiles = (chunks + kTileChunks - 1) / kTileChunks;
-    if (e == cudaSuccess) e = cudaMalloc((void**)&chunk, chunks * (sizeof(double) + sizeof(int32_t)) + tiles * sizeof(int32_t));
+    // chunk partials (double) followed by the chunk -> segment table (int32)
+    if (e == cudaSuccess) e = cudaMalloc((void**)&chunk, chunks * (sizeof(double) + sizeof(int32_t)));
     if (e == cudaSuccess) e = cudaMemset(base, 0, bytes);
     if (e == cudaSuccess) e = cudaMemset(chunk, 0, chunks * sizeof(double));
     if (e == cudaSuccess) e = cudaMemcpy(ctx->d_offsets, offsets, (B + 1) * sizeof(int64_t), cudaMemcpyHostToDevice);
@@ -1194,11 +1192,6 @@ int intsgd_set_blocks(intsgd_ctx* ctx, int32_t num_blocks, const int64_t* offset
         chunk_table_kernel<<<(unsigned)((chunks + 255) / 256), 256>>>(ctx->d_offsets, num_blocks, ctx->cfg.d,
                                                                       reinterpret_cast<int32_t*>(chunk + chunks), (int64_t)chunks);
         e = cudaGetLastError();
-        if (e == cudaSuccess) {
-            int32_t* seg_table = reinterpret_cast<int32_t*>(chunk + chunks);
-            tile_table_kernel<<<(unsigned)((tiles + 255) / 256), 256>>>(seg_table, (int64_t)chunks, seg_table + chunks, (int64_t)tiles);
-            e = cudaGetLastError();
-        }
         if (e == cudaSuccess) e = cudaDeviceSynchronize();
     }
     // covered ranges: whole units of 4 (direct kernels, fp32 pipelined) and pairs of units (bf16 pipelined)
@@ -1228,7 +1221,6 @@ int intsgd_set_blocks(intsgd_ctx* ctx, int32_t num_blocks, const int64_t* offset
     ctx->bs.c = ctx->bs.alpha + B;
     ctx->bs.chunk_sum = chunk;
     ctx->bs.chunk_seg = reinterpret_cast<int32_t*>(chunk + chunks);
-    ctx->bs.tile_seg = ctx->bs.chunk_seg + chunks;
     ctx->bs.B = num_blocks;
     return INTSGD_OK;
 }

@@ -71,28 +71,6 @@ __global__ void __launch_bounds__(256) chunk_table_kernel(const int64_t* offsets
     chunk_seg[k] = s | (crosses ? (int32_t)0x80000000 : 0);
 }
 
-// Table of whole tiles (32 chunks = 4096 coordinates): entry t is the segment of the tile if every chunk of it
-// that exists lies inside that one segment, else -1.  Built from the chunk table.
-constexpr int kTileChunks = 32;
-__global__ void __launch_bounds__(256) tile_table_kernel(const int32_t* chunk_seg, int64_t chunks, int32_t* tile_seg,
-                                                         int64_t tiles) {
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= tiles) return;
-    const int64_t k0 = t * kTileChunks;
-    int64_t k1 = k0 + kTileChunks - 1;
-    if (k1 > chunks - 1) k1 = chunks - 1;
-    const int32_t first = chunk_seg[k0], last = chunk_seg[k1];
-    // segments are contiguous: first and last chunk inside the same segment means all chunks between them are
-    tile_seg[t] = (first >= 0 && last == first) ? first : -1;
-}
-
-// (alpha, c) of tile t of the whole vector if the tile lies inside one segment, (NaN, 0) otherwise.
-__device__ __forceinline__ float2 tile_scale(const BlockParams& bp, int64_t t) {
-    const int32_t sg = __ldg(&bp.tile_seg[t]);
-    if (sg < 0) return make_float2(__int_as_float(0x7FC00000), 0.0f);
-    return make_float2(__ldg(&bp.alpha[sg]), __ldg(&bp.c[sg]));
-}
-
 __device__ __forceinline__ UnitScale unit_scale(const BlockParams& bp, int64_t unit, int s_lo, int s_hi) {
     UnitScale u;
     if (s_lo == s_hi) {
@@ -159,7 +137,6 @@ struct BlockState {
     float* c;           // B
     double* chunk_sum;
     const int32_t* chunk_seg;
-    const int32_t* tile_seg;
     double* edge_sum;
     double* tail_sq;
     int32_t B;

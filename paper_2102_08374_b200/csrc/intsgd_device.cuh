@@ -63,8 +63,6 @@ struct BlockParams {
     double* chunk_sum;        // device, ceil(d / 128)
     const int32_t* chunk_seg; // device, ceil(d / 128): segment of the chunk's first coordinate; sign bit set
                               // when the chunk's 128 coordinates reach into a later segment
-    const int32_t* tile_seg;  // device, ceil(d / 4096): the segment that holds all 4096 coordinates of the tile
-                              // (32 chunks, the tile of the pipelined kernels), or -1 if they are not in one segment
     double* edge_sum;         // device, B (cleared when the step opens)
     double* tail_sq;          // device, 8: squared steps of the coordinates after covered_end
     int64_t covered_end;      // coordinates below this are handled as whole units by the launch

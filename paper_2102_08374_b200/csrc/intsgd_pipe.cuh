@@ -74,18 +74,6 @@ __device__ __forceinline__ void drain_issued(uint64_t* full_bar, uint32_t issued
     }
 }
 
-// The tile's slice of the iterate is fetched when the tile starts and used when it ends.  As a volatile asm the
-// load keeps its place in front of the (volatile) barrier waits of the tile's stages: left to the compiler it may
-// be sunk to its use to save registers, which puts a full memory latency between two tiles.
-__device__ __forceinline__ float4 load_f4_early(const float* base, int64_t unit) {
-    float4 v;
-    asm volatile("ld.global.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "l"(reinterpret_cast<const float4*>(base) + unit)
-                 : "memory");
-    return v;
-}
-
 // ---- per-unit arithmetic ------------------------------------------------------------------------
 // Fast path of one worker's unit.  The rounded values are accumulated as integer-valued
 // floats (exact: the host caps the fast-path magnitude T so that n * (T + 1) <= 2^24, and T never
@@ -149,10 +137,6 @@ __device__ __noinline__ int4 redo_unit(const VecParams& P, int64_t unit, float4 
     return make_int4(S[0], S[1], S[2], S[3]);
 }
 
-// Tags of the two forms of the pipelined kernel's tile body.
-struct UniformTile { static constexpr bool value = true; };
-struct MixedTile { static constexpr bool value = false; };
-
 struct PipeParams {
     VecParams v;
     float fast_limit;   // T: fast path handles |alpha g| <= T
@@ -204,9 +188,6 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
     __shared__ uint64_t full_bar[NS], empty_bar[NS];
     __shared__ cnt_t s_cnt[INTSGD_MAX_WORKERS + 1];
     __shared__ int s_fault;
-    // Block-wise scales: (alpha, c) of the i-th tile of this block if the tile lies inside one segment, NaN otherwise.
-    constexpr int kTileCache = BLOCKS ? 2048 : 1;
-    __shared__ float2 s_tile_ac[kTileCache];
 
     const VecParams& P = PP.v;
     DevState* st = P.st;
@@ -229,18 +210,6 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
 
     const int n = P.n;
     const int64_t tiles = PP.tiles;
-    if (BLOCKS) {
-        // Almost every tile (4096 coordinates) lies inside one segment.  The scales of this block's tiles are
-        // staged in shared memory once, so that the steady state has no table look-up in flight between tiles.
-        static_assert(!BLOCKS || NC * UPT == 32 * kTileChunks, "the tile table is built for tiles of 32 chunks");
-        const int64_t tile_base = P.unit_base / (NC * UPT);   // a window starts on a tile boundary of the whole vector
-        for (int i = threadIdx.x; i < kTileCache; i += blockDim.x) {
-            const int64_t t = (int64_t)blockIdx.x + (int64_t)i * gridDim.x;
-            if (t >= tiles) break;
-            s_tile_ac[i] = tile_scale(P.bp, t + tile_base);
-        }
-        __syncthreads();
-    }
     ThreadAcc acc = {0.0, 0, 0u};
     bool ok = true;
     uint32_t it = 0;   // producer thread: stages filled so far
@@ -276,19 +245,29 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         uint32_t s = 0, phase = 0;
         float max_sum = 0.0f;                                            // max |S| over fast-path units
         const bool count_overflow = P.agg_limit != 0x7FFFFFFF;          // int8 wire: count |S| > 127
-        int tile_i = 0;   // index of the tile among this block's tiles
-        // One tile.  UNIFORM: all units of the tile take one scale pair (always with a scalar alpha; block-wise, a
-        // tile inside one segment): the body then holds no table look-up at all.  Otherwise every chunk looks its
-        // segment(s) up.  The two forms are separate copies of the body on purpose: a seldom-taken look-up inside
-        // the common body costs the common case several per cent.
-        auto tile_body = [&](const int64_t tile, const float2 tile_ac, auto uniform_tag) {
-            constexpr bool UNIFORM = decltype(uniform_tag)::value;
+        // Block-wise scales: the table entry of each of the thread's chunks and the scale of its first
+        // segment are fetched one tile ahead, so that no load sits between two tiles.
+        int32_t ent[UPT], ent_next[UPT];
+        float pre_a[UPT], pre_c[UPT];
+#pragma unroll
+        for (int k = 0; k < UPT; ++k) {
+            ent[k] = ent_next[k] = 0;
+            pre_a[k] = pre_c[k] = 0.0f;
+            if (BLOCKS) {
+                const int64_t chunk0 = (int64_t)blockIdx.x * kTileUnits + c + (int64_t)k * NC - lane;
+                if (chunk0 < PP.units) ent[k] = chunk_entry(bp, chunk0 + P.unit_base);
+                pre_a[k] = __ldg(&bp.alpha[ent[k] & 0x7FFFFFFF]);
+                pre_c[k] = __ldg(&bp.c[ent[k] & 0x7FFFFFFF]);
+            }
+        }
+        for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             const int64_t unit0 = tile * kTileUnits + c;
             float4 xo[UPT];
             PhiloxThreadPart tp[UPT];
             UnitAcc ua[UPT];
-            float2 a01[UPT];   // the scale of the unit's four coordinates (block-wise: of the chunk's first segment)
-            float ck[UPT];     // its decode factor
+            float2 a01[UPT], a23[UPT];
+            int s_lo[UPT], s_hi[UPT];
+            float c_uni[UPT];
             bool active[UPT], half[UPT];
 #pragma unroll
             for (int k = 0; k < UPT; ++k) {
@@ -296,7 +275,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 active[k] = unit < PP.units;
                 half[k] = ((unit + P.unit_base) >> 9) & 1;
                 xo[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (active[k]) xo[k] = load_f4_early(P.x, unit);
+                if (active[k]) xo[k] = load_f4<true>(P.x, unit);
                 tp[k].n3 = tp[k].H = tp[k].m1 = 0;
                 if (ROUND == INTSGD_ROUND_RANDOM || ROUND == INTSGD_ROUND_RANDOM_COMPARE)
                     tp[k] = philox_thread_part((uint32_t)(unit + P.unit_base), step, P.keys);
@@ -305,20 +284,32 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 ua[k].F01 = make_float2(0.f, 0.f);
                 ua[k].F23 = make_float2(0.f, 0.f);
                 ua[k].m = 0.0f;
-                a01[k] = make_float2(tile_ac.x, tile_ac.x);
-                ck[k] = tile_ac.y;
-                if (!UNIFORM && unit - lane < PP.units) {
-                    // The warp's 32 units form one chunk.  The fast path rounds with the scale of the chunk's first
-                    // segment; a chunk that reaches into another segment (rare: at most two per boundary) discards
-                    // that work and is redone coordinate by coordinate at the end of the tile.
-                    const int sg = chunk_entry(bp, unit - lane + P.unit_base) & 0x7FFFFFFF;
-                    const float a = __ldg(&bp.alpha[sg]);
-                    a01[k] = make_float2(a, a);
-                    ck[k] = __ldg(&bp.c[sg]);
+                a01[k] = make_float2(alpha, alpha);
+                a23[k] = a01[k];
+                s_lo[k] = s_hi[k] = 0;
+                c_uni[k] = 0.0f;
+                if (BLOCKS) {
+                    // the warp's 32 units form one chunk; chunks past the covered range are never committed
+                    if (unit - lane < PP.units) chunk_segments_from(bp, ent[k], unit - lane + P.unit_base, s_lo[k], s_hi[k]);
+                    if (active[k]) {
+                        if (s_lo[k] == s_hi[k]) {   // the chunk lies in one segment: scale and decode factor are at hand
+                            a01[k] = make_float2(pre_a[k], pre_a[k]);
+                            a23[k] = a01[k];
+                            c_uni[k] = pre_c[k];
+                        } else {
+                            const UnitScale us = unit_scale(bp, unit + P.unit_base, s_lo[k], s_hi[k]);
+                            a01[k] = us.a01;
+                            a23[k] = us.a23;
+                        }
+                    }
+                    const int64_t next_chunk0 = unit - lane + (int64_t)gridDim.x * kTileUnits;
+                    ent_next[k] = (next_chunk0 < PP.units) ? chunk_entry(bp, next_chunk0 + P.unit_base) : 0;
                 }
             }
             for (int g0 = 0; g0 < n; g0 += G) {
-                if (!mbar_wait(&full_bar[s], phase)) { ok = false; break; }
+                bool arrived = mbar_wait(&full_bar[s], phase);
+                if (BLOCKS) arrived = __all_sync(0xFFFFFFFFu, arrived);   // keep the warp together for the shuffles below
+                if (!arrived) { ok = false; break; }
                 const unsigned char* src = smem + (size_t)s * G * kTileBytes;
                 const int gw = (n - g0 < G) ? (n - g0) : G;
                 if (active[UPT - 1] && gw == G) {
@@ -331,7 +322,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
 #pragma unroll
                         for (int k = 0; k < UPT; ++k) {
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
-                            consume_unit<ROUND>(gv, a01[k], a01[k], unit_draws<ROUND, kPairShared>(tp[k], e, pw, k, half[k], P.keys), ua[k]);
+                            consume_unit<ROUND>(gv, a01[k], a23[k], unit_draws<ROUND, kPairShared>(tp[k], e, pw, k, half[k], P.keys), ua[k]);
                         }
                     }
                 } else {
@@ -343,63 +334,62 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                         for (int k = 0; k < UPT; ++k) {
                             if (!active[k]) continue;
                             const float4 gv = lds_unit<GRAD>(src + w * kTileBytes, c + k * NC);
-                            consume_unit<ROUND>(gv, a01[k], a01[k], unit_draws<ROUND, kPairShared>(tp[k], e, pw, k, half[k], P.keys), ua[k]);
+                            consume_unit<ROUND>(gv, a01[k], a23[k], unit_draws<ROUND, kPairShared>(tp[k], e, pw, k, half[k], P.keys), ua[k]);
                         }
                     }
                 }
                 mbar_arrive(&empty_bar[s]);
                 if (++s == NS) { s = 0; phase ^= 1u; }
             }
-            // A wait that gave up (ok == false) ends the kernel after this tile.  Block-wise, every lane still walks
-            // the epilogue, so that the warp's shuffles below stay complete; nothing of a failed tile is stored.
-            if (!BLOCKS && !ok) return;
-            double chunk_sq[UPT];   // block-wise: this lane's share of its chunks' squared step lengths
-            bool chunk_done[UPT];   // the chunk exists and lies in one segment: its partial goes to chunk_sum
+            if (!ok) break;
+            float next_a[UPT], next_c[UPT];
 #pragma unroll
             for (int k = 0; k < UPT; ++k) {
-                chunk_sq[k] = 0.0;
-                chunk_done[k] = false;
+                next_a[k] = next_c[k] = 0.0f;
+                if (BLOCKS) {   // the entries have arrived during the tile; these two loads overlap the epilogue
+                    next_a[k] = __ldg(&bp.alpha[ent_next[k] & 0x7FFFFFFF]);
+                    next_c[k] = __ldg(&bp.c[ent_next[k] & 0x7FFFFFFF]);
+                }
             }
 #pragma unroll
             for (int k = 0; k < UPT; ++k) {
                 const int64_t unit = unit0 + (int64_t)k * NC;
                 if (BLOCKS) {
                     if (unit - lane >= PP.units) continue;   // warp-uniform: this chunk does not exist
-                    int s_lo = 0, s_hi = 0;   // equal: the chunk lies in one segment (its index is not needed then)
-                    if (!UNIFORM) chunk_segments(bp, unit - lane + P.unit_base, s_lo, s_hi);
-                    if (s_lo != s_hi) {
-                        // the chunk crosses a segment boundary: per-coordinate scales from global memory, one partial
-                        // per segment
+                    if (s_lo[k] != s_hi[k]) {
+                        // the chunk crosses a segment boundary: per-coordinate scales, one partial per segment
                         double sq[4] = {0.0, 0.0, 0.0, 0.0};
                         int seg[4] = {-1, -1, -1, -1};
                         if (active[k]) {
-                            const UnitScale us = unit_scale(bp, unit + P.unit_base, s_lo, s_hi);
-                            const int4 S = redo_unit<GRAD, ROUND>(P, unit, make_float4(us.a01.x, us.a01.y, us.a23.x, us.a23.y), step, s_cnt);
+                            const UnitScale us = unit_scale(bp, unit + P.unit_base, s_lo[k], s_hi[k]);
+                            int4 S;
+                            if (ua[k].m <= PP.fast_limit)
+                                S = make_int4(__float2int_rn(ua[k].F01.x), __float2int_rn(ua[k].F01.y),
+                                              __float2int_rn(ua[k].F23.x), __float2int_rn(ua[k].F23.y));
+                            else
+                                S = redo_unit<GRAD, ROUND>(P, unit, make_float4(us.a01.x, us.a01.y, us.a23.x, us.a23.y), step, s_cnt);
                             float4 xn;
                             xn.x = update_coord_sq(xo[k].x, __int2float_rn(S.x), us.c.x, sq[0]);
                             xn.y = update_coord_sq(xo[k].y, __int2float_rn(S.y), us.c.y, sq[1]);
                             xn.z = update_coord_sq(xo[k].z, __int2float_rn(S.z), us.c.z, sq[2]);
                             xn.w = update_coord_sq(xo[k].w, __int2float_rn(S.w), us.c.w, sq[3]);
-                            if (ok) {
-                                store_f4<true>(P.x, unit, xn);
-                                if (P.agg) store_i4<true>(P.agg, unit, S);
-                            }
+                            store_f4<true>(P.x, unit, xn);
+                            if (P.agg) store_i4<true>(P.agg, unit, S);
                             note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
                             note_sum(S.z, P.agg_limit, acc); note_sum(S.w, P.agg_limit, acc);
 #pragma unroll
                             for (int e = 0; e < 4; ++e) seg[e] = us.seg[e];
                         }
-                        chunk_commit(bp, unit - lane + P.unit_base, s_lo, s_hi, sq, seg);
+                        chunk_commit(bp, unit - lane + P.unit_base, s_lo[k], s_hi[k], sq, seg);
                         continue;
                     }
                 } else if (!active[k]) {
                     continue;
                 }
                 // One scale for the whole unit (always, or a chunk inside one segment).
-                chunk_done[k] = true;
                 double unit_sq = 0.0;   // squared step of the unit: ((d0^2 + d1^2) + d2^2) + d3^2, products exact
                 if (active[k]) {
-                    const float cu = ck[k];
+                    const float cu = BLOCKS ? c_uni[k] : cdec;
                     int4 S;
                     float2 S01, S23;   // the sums as floats (exact on the fast path)
                     if (ua[k].m <= PP.fast_limit) {
@@ -412,7 +402,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                             acc.overflow += (fabsf(S01.x) > 127.0f) + (fabsf(S01.y) > 127.0f) + (fabsf(S23.x) > 127.0f) +
                                             (fabsf(S23.y) > 127.0f);
                     } else {
-                        S = redo_unit<GRAD, ROUND>(P, unit, make_float4(a01[k].x, a01[k].x, a01[k].x, a01[k].x), step, s_cnt);
+                        S = redo_unit<GRAD, ROUND>(P, unit, make_float4(a01[k].x, a01[k].y, a23[k].x, a23[k].y), step, s_cnt);
                         S01 = make_float2(__int2float_rn(S.x), __int2float_rn(S.y));
                         S23 = make_float2(__int2float_rn(S.z), __int2float_rn(S.w));
                         note_sum(S.x, P.agg_limit, acc); note_sum(S.y, P.agg_limit, acc);
@@ -429,38 +419,19 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                     *sink = __fma_rn((double)d01.y, (double)d01.y, *sink);
                     *sink = __fma_rn((double)d23.x, (double)d23.x, *sink);
                     *sink = __fma_rn((double)d23.y, (double)d23.y, *sink);
-                    if (!BLOCKS || ok) {
-                        store_f4<true>(P.x, unit, make_float4(xn01.x, xn01.y, xn23.x, xn23.y));
-                        if (P.agg) store_i4<true>(P.agg, unit, S);
-                    }
+                    store_f4<true>(P.x, unit, make_float4(xn01.x, xn01.y, xn23.x, xn23.y));
+                    if (P.agg) store_i4<true>(P.agg, unit, S);
                 }
-                if (BLOCKS) chunk_sq[k] = unit_sq;
+                if (BLOCKS) {   // all 32 lanes of the warp: one partial per chunk, fixed order
+                    const double t = warp_tree(unit_sq);
+                    if (lane == 0) __stcg(&bp.chunk_sum[(unit - lane + P.unit_base) >> 5], t);
+                }
             }
-            if (BLOCKS) {
-                // One partial per chunk, summed over the warp's 32 units in a fixed order; the UPT trees advance level
-                // by level together, so that their shuffle latencies overlap.
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) {
-#pragma unroll
-                    for (int k = 0; k < UPT; ++k) chunk_sq[k] += __shfl_down_sync(0xFFFFFFFFu, chunk_sq[k], off);
-                }
-#pragma unroll
-                for (int k = 0; k < UPT; ++k) {
-                    const int64_t chunk_unit0 = unit0 + (int64_t)k * NC - lane;
-                    if (lane == 0 && chunk_done[k] && ok) __stcg(&bp.chunk_sum[(chunk_unit0 + P.unit_base) >> 5], chunk_sq[k]);
-                }
-                ok = __all_sync(0xFFFFFFFFu, ok);   // the warp leaves the tile loop together
-            }
-        };
-        for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-            if (!BLOCKS) {
-                tile_body(tile, make_float2(alpha, cdec), UniformTile());
-            } else {
-                // NaN marks a tile that is not inside one segment; tiles beyond the staged table take the same path
-                const float2 tile_ac = tile_i < kTileCache ? s_tile_ac[tile_i] : make_float2(__int_as_float(0x7FC00000), 0.0f);
-                ++tile_i;
-                if (tile_ac.x == tile_ac.x) tile_body(tile, tile_ac, UniformTile());
-                else tile_body(tile, make_float2(0.0f, 0.0f), MixedTile());
+            for (int k = 0; k < UPT; ++k) {
+                ent[k] = ent_next[k];
+                pre_a[k] = next_a[k];
+                pre_c[k] = next_c[k];
             }
         }
         {   // fold the float-tracked maximum of the fast-path sums (integers below 2^24) into the counters
