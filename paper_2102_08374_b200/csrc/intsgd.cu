@@ -161,6 +161,23 @@ int after_launch(intsgd_ctx* ctx, const char* what) {
 
 // ---- launchers -------------------------------------------------------------------------
 
+// Launch as a programmatic dependent of the kernel in front of it on the stream: the grid may become resident
+// while that kernel drains (its launch latency leaves the step's path); every kernel launched this way executes
+// griddepcontrol.wait before it touches memory the kernel in front writes.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 int launch_scale(intsgd_ctx* ctx, double eta, double dx2_override, cudaStream_t s) {
     if (!(eta > 0.0) || !std::isfinite(eta)) return fail(ctx, INTSGD_ERR_INVALID_ARG, "eta_k must be finite and > 0");
     if (std::isnan(dx2_override) || std::isinf(dx2_override))
@@ -169,8 +186,9 @@ int launch_scale(intsgd_ctx* ctx, double eta, double dx2_override, cudaStream_t 
     if (ctx->bs.B > 0) {
         if (dx2_override >= 0.0)
             return fail(ctx, INTSGD_ERR_UNSUPPORTED, "dx2_override is not available with block-wise scales");
-        scale_blocks_kernel<<<1, 1024, 0, s>>>(ctx->d_state, ctx->bs, dd, 2.0 * dn, dn, eta, ctx->cfg.beta, ctx->cfg.eps,
-                                               ctx->cfg.n);
+        const cudaError_t e = launch_dependent(scale_blocks_kernel, dim3(1), dim3(1024), s, ctx->d_state, ctx->bs, dd, 2.0 * dn, dn,
+                                               eta, ctx->cfg.beta, ctx->cfg.eps, (int32_t)ctx->cfg.n);
+        if (e != cudaSuccess) return fail(ctx, INTSGD_ERR_CUDA, "launch of scale_blocks_kernel failed: %s", cudaGetErrorString(e));
         return after_launch(ctx, "scale_blocks_kernel");
     }
     // The scale kernel may be scheduled while the kernel before it on the stream is still running (it waits
@@ -427,12 +445,15 @@ int launch_block_norm(intsgd_ctx* ctx, int64_t covered_end, bool check_status, b
     const NormPlan& plan = (ctx->plan[0].covered_end == covered_end) ? ctx->plan[0] : ctx->plan[1];
     if (plan.covered_end != covered_end) return fail(ctx, INTSGD_ERR_CUDA, "internal: no reduction plan for this launch");
     if (plan.num_slices > 0) {
-        block_norm_slices_kernel<<<plan.num_slices, 256, 0, s>>>(ctx->d_state, ctx->bs, plan, check_status ? 1 : 0);
+        const cudaError_t e = launch_dependent(block_norm_slices_kernel, dim3(plan.num_slices), dim3(256), s,
+                                               (const DevState*)ctx->d_state, ctx->bs, plan, (int32_t)(check_status ? 1 : 0));
+        if (e != cudaSuccess) return fail(ctx, INTSGD_ERR_CUDA, "launch of block_norm_slices_kernel failed: %s", cudaGetErrorString(e));
         const int rc = after_launch(ctx, "block_norm_slices_kernel");
         if (rc != INTSGD_OK) return rc;
     }
-    block_norm_kernel<<<ctx->bs.B, 128, 0, s>>>(ctx->d_state, ctx->bs, plan, ctx->cfg.d, check_status ? 1 : 0,
-                                                advance_step ? 1 : 0);
+    const cudaError_t e = launch_dependent(block_norm_kernel, dim3(ctx->bs.B), dim3(128), s, ctx->d_state, ctx->bs, plan,
+                                           (int64_t)ctx->cfg.d, (int32_t)(check_status ? 1 : 0), (int32_t)(advance_step ? 1 : 0));
+    if (e != cudaSuccess) return fail(ctx, INTSGD_ERR_CUDA, "launch of block_norm_kernel failed: %s", cudaGetErrorString(e));
     return after_launch(ctx, "block_norm_kernel");
 }
 

@@ -150,6 +150,7 @@ __global__ void __launch_bounds__(1024) scale_blocks_kernel(DevState* st, BlockS
                                                             double n_as_double, double eta, double beta, double eps,
                                                             int32_t n) {
     asm volatile("griddepcontrol.launch_dependents;");   // see scale_kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // the per-block norms of the step in front
     int bad = 0;
     for (int l = threadIdx.x; l < bs.B; l += blockDim.x) {
         const double dl = (double)(bs.offsets[l + 1] - bs.offsets[l]);
@@ -205,6 +206,10 @@ struct NormPlan {
 __global__ void __launch_bounds__(256) block_norm_slices_kernel(const DevState* st, BlockState bs, NormPlan plan,
                                                                 int32_t check_status) {
     __shared__ double s_warp[32];
+    // launched as a programmatic dependent of the step's vector kernel: may be resident early, reads nothing before
+    // that kernel has completed; its own dependent (pass 2) may be scheduled at once
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (check_status && st->status != INTSGD_OK) return;
     const int w = blockIdx.x;
     double v = 0.0;
@@ -220,6 +225,8 @@ __global__ void __launch_bounds__(128) block_norm_kernel(DevState* st, BlockStat
                                                          int32_t check_status, int32_t advance_step) {
     __shared__ double s_warp[32];
     __shared__ bool s_last;
+    asm volatile("griddepcontrol.launch_dependents;");   // the next step's scale kernel; it waits for this grid
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // pass 1 (or the vector kernel) has completed
     if (check_status && st->status != INTSGD_OK) return;
     const int l = blockIdx.x;
     double v = 0.0;
