@@ -33,14 +33,28 @@ METRIC = "fused IntSGD step throughput"
 UNIT = "gradient elements/s"
 HBM_FALLBACK_GBS = 6650.0
 
-# DRAM traffic of the fused kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum;
-# command and figures in profiles/fused_pipe_kernel_d24_n16_ncu_full.md): bytes per coordinate of the
-# captured case (d = 2^24, n = 16, fp32, int32 aggregate), valid for the kernel sources with this hash.
-# Any change to the kernel sources makes `roofline.traffic` null until the counters are taken again.
-NCU_TRAFFIC = {"sources_sha256": "814cfb67602a3a7f3fbd42e8e07cfa2ef11b35b2e45f9a2587e92c90d0795469",
-               "bytes_per_coordinate": 1.266082e9 / (1 << 24), "workers": 16, "grad": "f32", "mode": "fused",
-               # smsp__inst_executed.sum of the same capture: warp instructions per launch -> thread instructions per element
-               "instructions_per_element": 136.115e6 * 32 / (16 * (1 << 24))}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) and executed warp instructions of the kernels of one
+# step, from ncu captures of the small case (d = 2^24) of each shape this script can time; both grow in proportion
+# to d, so a launch at another d is the per-coordinate figure times d.  Valid for the kernel sources with this hash:
+# any change to them makes `roofline.traffic` null until the counters are taken again.
+NCU_COUNTERS = {
+    "sources_sha256": "e688988e442a68a0e979f2be54c29c4eaec860029bbec3bbaabef8cacf433c44",
+    "captured_log2d": 24,
+    # key: kind/mode/grad/payload/n -> bytes per coordinate, warp instructions per coordinate (the vector kernels of a
+    # step: fused; encode + aggregate; IntDIANA; block-wise (62 blocks); profiling pass + fused (16 bits))
+    "shapes": {
+        "intsgd/fused/f32/int32/n16": {"bytes_per_coordinate": 75.401, "warp_instructions_per_coordinate": 8.1142},
+        "intsgd/fused/f32/int32/n8": {"bytes_per_coordinate": 42.79, "warp_instructions_per_coordinate": 4.3565},
+        "intsgd/fused/f32/int32/n2": {"bytes_per_coordinate": 16.978, "warp_instructions_per_coordinate": 2.0196},
+        "intsgd/fused/bf16/int8/n8": {"bytes_per_coordinate": 25.982, "warp_instructions_per_coordinate": 4.4747},
+        "intsgd/two_kernel/f32/int32/n16": {"bytes_per_coordinate": 197.99, "warp_instructions_per_coordinate": 9.8815},
+        "intsgd/two_kernel/f32/int8/n16": {"bytes_per_coordinate": 103.678, "warp_instructions_per_coordinate": 10.0865},
+        "intsgd/two_kernel/bf16/int8/n8": {"bytes_per_coordinate": 38.597, "warp_instructions_per_coordinate": 5.3433},
+        "diana/fused/f32/int32/n16": {"bytes_per_coordinate": 209.324, "warp_instructions_per_coordinate": 16.069},
+        "blocks/fused/f32/int32/n16": {"bytes_per_coordinate": 75.483, "warp_instructions_per_coordinate": 9.2801},
+        "heuristic/fused/f32/int32/n16": {"bytes_per_coordinate": 139.592, "warp_instructions_per_coordinate": 9.1813},
+    },
+}
 
 
 def kernel_sources_hash():
@@ -52,14 +66,25 @@ def kernel_sources_hash():
     return h.hexdigest()
 
 
-def traffic_per_launch(args, d):
-    """Measured DRAM bytes per launch, scaled to d (traffic is proportional to d), or None."""
-    t = NCU_TRAFFIC
-    same = (args.workers == t["workers"] and args.grad == t["grad"] and args.mode == t["mode"]
-            and args.rounding == "random" and args.kind == "intsgd")
-    if not same or kernel_sources_hash() != t["sources_sha256"]:
+def shape_key(args):
+    return f"{args.kind}/{args.mode}/{args.grad}/{args.payload}/n{args.workers}"
+
+
+def captured_counters(args):
+    """The ncu figures of this shape (default random stream only), or None."""
+    if args.rounding != "random" or kernel_sources_hash() != NCU_COUNTERS["sources_sha256"]:
         return None
-    return t["bytes_per_coordinate"] * d
+    if args.kind == "blocks" and args.num_blocks != 62:
+        return None
+    if args.kind == "heuristic" and args.num_bits != 16:
+        return None
+    return NCU_COUNTERS["shapes"].get(shape_key(args))
+
+
+def traffic_per_launch(args, d):
+    """Measured DRAM bytes of one step's kernels, scaled to d (traffic is proportional to d), or None."""
+    c = captured_counters(args)
+    return None if c is None else c["bytes_per_coordinate"] * d
 
 
 def parse_args():
@@ -490,6 +515,10 @@ def main():
                 "sustained": sustained}
     if clocks.get("sm_mhz"):
         roofline["sm_clocks_per_worker_unit"] = avg_ms * 1e-3 * clocks["sm_mhz"] * 1e6 * sms / (n * d / 4)
+    counters = captured_counters(args)
+    if counters is not None:
+        roofline["traffic_over_algorithmic"] = counters["bytes_per_coordinate"] * d / bytes_per_launch
+        roofline["thread_instructions_per_element"] = counters["warp_instructions_per_coordinate"] * 32 / n
 
     # ---- second limit: the 32x32->64-bit multiplies of Philox4x32-10, against their rate measured alone ----
     mults = wide_multiplies_per_worker_unit(args, n)
