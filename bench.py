@@ -38,21 +38,21 @@ HBM_FALLBACK_GBS = 6650.0
 # to d, so a launch at another d is the per-coordinate figure times d.  Valid for the kernel sources with this hash:
 # any change to them makes `roofline.traffic` null until the counters are taken again.
 NCU_COUNTERS = {
-    "sources_sha256": "e688988e442a68a0e979f2be54c29c4eaec860029bbec3bbaabef8cacf433c44",
+    "sources_sha256": "ae5959cc4c17eed55c1cd416055a97961362b01f850dcf15de37fe945b28a3b5",
     "captured_log2d": 24,
     # key: kind/mode/grad/payload/n -> bytes per coordinate, warp instructions per coordinate (the vector kernels of a
     # step: fused; encode + aggregate; IntDIANA; block-wise (62 blocks); profiling pass + fused (16 bits))
     "shapes": {
-        "intsgd/fused/f32/int32/n16": {"bytes_per_coordinate": 75.401, "warp_instructions_per_coordinate": 8.1142},
-        "intsgd/fused/f32/int32/n8": {"bytes_per_coordinate": 42.79, "warp_instructions_per_coordinate": 4.3565},
-        "intsgd/fused/f32/int32/n2": {"bytes_per_coordinate": 16.978, "warp_instructions_per_coordinate": 2.0196},
-        "intsgd/fused/bf16/int8/n8": {"bytes_per_coordinate": 25.982, "warp_instructions_per_coordinate": 4.4747},
-        "intsgd/two_kernel/f32/int32/n16": {"bytes_per_coordinate": 197.99, "warp_instructions_per_coordinate": 9.8815},
-        "intsgd/two_kernel/f32/int8/n16": {"bytes_per_coordinate": 103.678, "warp_instructions_per_coordinate": 10.0865},
-        "intsgd/two_kernel/bf16/int8/n8": {"bytes_per_coordinate": 38.597, "warp_instructions_per_coordinate": 5.3433},
-        "diana/fused/f32/int32/n16": {"bytes_per_coordinate": 209.324, "warp_instructions_per_coordinate": 16.069},
-        "blocks/fused/f32/int32/n16": {"bytes_per_coordinate": 75.483, "warp_instructions_per_coordinate": 9.2801},
-        "heuristic/fused/f32/int32/n16": {"bytes_per_coordinate": 139.592, "warp_instructions_per_coordinate": 9.1813},
+        "intsgd/fused/f32/int32/n16": {"bytes_per_coordinate": 75.393, "warp_instructions_per_coordinate": 8.1141},
+        "intsgd/fused/f32/int32/n8": {"bytes_per_coordinate": 42.904, "warp_instructions_per_coordinate": 4.3562},
+        "intsgd/fused/f32/int32/n2": {"bytes_per_coordinate": 16.955, "warp_instructions_per_coordinate": 2.0197},
+        "intsgd/fused/bf16/int8/n8": {"bytes_per_coordinate": 26.06, "warp_instructions_per_coordinate": 4.4747},
+        "intsgd/two_kernel/f32/int32/n16": {"bytes_per_coordinate": 197.936, "warp_instructions_per_coordinate": 9.8816},
+        "intsgd/two_kernel/f32/int8/n16": {"bytes_per_coordinate": 103.557, "warp_instructions_per_coordinate": 10.754},
+        "intsgd/two_kernel/bf16/int8/n8": {"bytes_per_coordinate": 38.428, "warp_instructions_per_coordinate": 5.7685},
+        "diana/fused/f32/int32/n16": {"bytes_per_coordinate": 209.336, "warp_instructions_per_coordinate": 16.07},
+        "blocks/fused/f32/int32/n16": {"bytes_per_coordinate": 75.581, "warp_instructions_per_coordinate": 9.2814},
+        "heuristic/fused/f32/int32/n16": {"bytes_per_coordinate": 139.591, "warp_instructions_per_coordinate": 9.1813},
     },
 }
 

@@ -297,7 +297,7 @@ int launch_aggregate(intsgd_ctx* ctx, const VecParams& P, bool aligned, cudaStre
         if (rc != INTSGD_OK) return rc;
         return launch_block_norm(ctx, covered, true, true, s);
     }
-    const int64_t items = (i8 && aligned) ? (ctx->cfg.d + 15) / 16 : (i8 ? ctx->cfg.d : (ctx->cfg.d + 3) / 4);
+    const int64_t items = (i8 && !aligned) ? ctx->cfg.d : (ctx->cfg.d + 3) / 4;
     const int grid = grid_for(ctx, items);
     if (!i8 && aligned) aggregate_kernel<INTSGD_PAYLOAD_I32, true><<<grid, ctx->threads, 0, s>>>(P);
     else if (!i8) aggregate_kernel<INTSGD_PAYLOAD_I32, false><<<grid, ctx->threads, 0, s>>>(P);

@@ -140,8 +140,8 @@ __global__ void __launch_bounds__(kMaxThreads) encode_kernel(const __grid_consta
 
 // ----------------------------------------------------------------------------------------
 // Aggregate + decode + update + next-norm partial, one pass.
-// int32 payloads: one unit (4 coordinates) per thread iteration.
-// int8 payloads : four units (16 coordinates, one 16-byte load per worker) per iteration.
+// One unit (4 coordinates) per thread iteration: a 16-byte load per worker on the int32 wire, one packed 32-bit
+// word per worker on the int8 wire.
 // ----------------------------------------------------------------------------------------
 template <bool ALIGNED>
 __device__ __forceinline__ void apply_unit(const VecParams& P, int64_t unit, int4 S, float c, ThreadAcc& acc) {
@@ -187,29 +187,24 @@ __global__ void __launch_bounds__(kMaxThreads) aggregate_kernel(const __grid_con
             apply_unit<ALIGNED>(P, unit, S, c, acc);
         }
         done = full << 2;
-    } else {
-        const int64_t full16 = ALIGNED ? (P.d >> 4) : 0;
-        for (int64_t u16 = first; u16 < full16; u16 += stride) {
-            int4 S0 = make_int4(0, 0, 0, 0), S1 = S0, S2 = S0, S3 = S0;
-#pragma unroll 4
-            for (int i = 0; i < n; ++i) {
-                const uint4 v = __ldcs((const uint4*)P.in[i] + u16);
-                add_bytes(S0, v.x); add_bytes(S1, v.y); add_bytes(S2, v.z); add_bytes(S3, v.w);
-            }
-            apply_unit<ALIGNED>(P, 4 * u16 + 0, S0, c, acc);
-            apply_unit<ALIGNED>(P, 4 * u16 + 1, S1, c, acc);
-            apply_unit<ALIGNED>(P, 4 * u16 + 2, S2, c, acc);
-            apply_unit<ALIGNED>(P, 4 * u16 + 3, S3, c, acc);
+    } else if (ALIGNED) {
+        // int8 wire: one unit = one packed 32-bit word per worker; consecutive lanes take consecutive units, so every
+        // access of a warp (payload words, x, aggregate) is one contiguous run
+        const int64_t full = P.d >> 2;
+        for (int64_t unit = first; unit < full; unit += stride) {
+            int4 S = make_int4(0, 0, 0, 0);
+#pragma unroll 8
+            for (int i = 0; i < n; ++i) add_bytes(S, __ldcs((const uint32_t*)P.in[i] + unit));
+            apply_unit<ALIGNED>(P, unit, S, c, acc);
         }
-        done = full16 << 4;
-        if (!ALIGNED) {   // element-wise path for unaligned int8 payloads
-            for (int64_t j = first; j < P.d; j += stride) {
-                int S = 0;
-                for (int i = 0; i < n; ++i) S += (int)((const int8_t*)P.in[i])[j];
-                apply_coord(P, j, S, c, acc);
-            }
-            done = P.d;
+        done = full << 2;
+    } else {   // element-wise path for unaligned int8 payloads
+        for (int64_t j = first; j < P.d; j += stride) {
+            int S = 0;
+            for (int i = 0; i < n; ++i) S += (int)((const int8_t*)P.in[i])[j];
+            apply_coord(P, j, S, c, acc);
         }
+        done = P.d;
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         for (int64_t j = done; j < P.d; ++j) {
