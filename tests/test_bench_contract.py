@@ -46,3 +46,34 @@ def test_algorithmic_bytes_per_coordinate():
     assert f(16, 4, 4, "fused", "diana") == 12 * 16 + 20
     assert f(16, 4, 4, "fused", "heuristic") == 2 * 64 + 12
     assert f(16, 4, 4, "fused", "blocks") == 76
+
+
+def test_counter_table_and_multiply_counts():
+    """The ncu counter table is keyed by shape, scales with d, and goes silent for anything it was not taken on."""
+    sys.path.insert(0, str(ROOT))
+    import argparse
+    import bench
+    base = dict(kind="intsgd", mode="fused", grad="f32", payload="int32", workers=16, rounding="random",
+                num_blocks=62, num_bits=16)
+    args = argparse.Namespace(**base)
+    assert bench.shape_key(args) == "intsgd/fused/f32/int32/n16"
+    fresh = bench.kernel_sources_hash() == bench.NCU_COUNTERS["sources_sha256"]
+    t = bench.traffic_per_launch(args, 1 << 26)
+    if fresh:   # counters taken on these very sources: traffic is within a few per cent of the algorithmic bytes
+        assert t is not None and abs(t / (76 * (1 << 26)) - 1.0) < 0.05
+        assert bench.traffic_per_launch(args, 1 << 28) == 4 * t
+    else:       # the kernels changed since the capture: no stale figure is reported
+        assert t is None
+    for other in (dict(rounding="compare"), dict(workers=5), dict(kind="blocks", num_blocks=7)):
+        assert bench.traffic_per_launch(argparse.Namespace(**{**base, **other}), 1 << 26) is None
+    for key, v in bench.NCU_COUNTERS["shapes"].items():
+        kind, mode, grad, payload, n = key.split("/")
+        n = int(n[1:])
+        gb, pb = (2 if grad == "bf16" else 4), (1 if payload == "int8" else 4)
+        alg = bench.algorithmic_bytes_per_coordinate(n, gb, pb, mode, kind)
+        # never above the algorithmic bytes (no stream is read twice); below them by what is still in L2 at kernel end
+        assert 0.8 < v["bytes_per_coordinate"] / alg < 1.02, key
+    # 32x32->64-bit products of the random stream per worker unit on the pipelined kernels
+    f = bench.wide_multiplies_per_worker_unit
+    assert f(argparse.Namespace(rounding="random"), 16) == 16.125 and f(argparse.Namespace(rounding="compare"), 8) == 16.25
+    assert f(argparse.Namespace(rounding="random16"), 16) == 8.0625 and f(argparse.Namespace(rounding="nearest"), 16) == 0.0
