@@ -38,21 +38,21 @@ HBM_FALLBACK_GBS = 6650.0
 # to d, so a launch at another d is the per-coordinate figure times d.  Valid for the kernel sources with this hash:
 # any change to them makes `roofline.traffic` null until the counters are taken again.
 NCU_COUNTERS = {
-    "sources_sha256": "ae5959cc4c17eed55c1cd416055a97961362b01f850dcf15de37fe945b28a3b5",
+    "sources_sha256": "f7138ccd759701a69cd46cff8b9acfeedf0ea0795dd26f55554882b8a1fbb780",
     "captured_log2d": 24,
     # key: kind/mode/grad/payload/n -> bytes per coordinate, warp instructions per coordinate (the vector kernels of a
     # step: fused; encode + aggregate; IntDIANA; block-wise (62 blocks); profiling pass + fused (16 bits))
     "shapes": {
-        "intsgd/fused/f32/int32/n16": {"bytes_per_coordinate": 75.393, "warp_instructions_per_coordinate": 8.1141},
-        "intsgd/fused/f32/int32/n8": {"bytes_per_coordinate": 42.904, "warp_instructions_per_coordinate": 4.3562},
-        "intsgd/fused/f32/int32/n2": {"bytes_per_coordinate": 16.955, "warp_instructions_per_coordinate": 2.0197},
-        "intsgd/fused/bf16/int8/n8": {"bytes_per_coordinate": 26.06, "warp_instructions_per_coordinate": 4.4747},
-        "intsgd/two_kernel/f32/int32/n16": {"bytes_per_coordinate": 197.936, "warp_instructions_per_coordinate": 9.8816},
-        "intsgd/two_kernel/f32/int8/n16": {"bytes_per_coordinate": 103.557, "warp_instructions_per_coordinate": 10.754},
-        "intsgd/two_kernel/bf16/int8/n8": {"bytes_per_coordinate": 38.428, "warp_instructions_per_coordinate": 5.7685},
-        "diana/fused/f32/int32/n16": {"bytes_per_coordinate": 209.336, "warp_instructions_per_coordinate": 16.07},
-        "blocks/fused/f32/int32/n16": {"bytes_per_coordinate": 75.581, "warp_instructions_per_coordinate": 9.2814},
-        "heuristic/fused/f32/int32/n16": {"bytes_per_coordinate": 139.591, "warp_instructions_per_coordinate": 9.1813},
+        "intsgd/fused/f32/int32/n16": {"bytes_per_coordinate": 75.39, "warp_instructions_per_coordinate": 8.1141},
+        "intsgd/fused/f32/int32/n8": {"bytes_per_coordinate": 42.9, "warp_instructions_per_coordinate": 4.3565},
+        "intsgd/fused/f32/int32/n2": {"bytes_per_coordinate": 16.997, "warp_instructions_per_coordinate": 2.0197},
+        "intsgd/fused/bf16/int8/n8": {"bytes_per_coordinate": 25.991, "warp_instructions_per_coordinate": 4.4747},
+        "intsgd/two_kernel/f32/int32/n16": {"bytes_per_coordinate": 197.937, "warp_instructions_per_coordinate": 9.8853},
+        "intsgd/two_kernel/f32/int8/n16": {"bytes_per_coordinate": 103.639, "warp_instructions_per_coordinate": 10.754},
+        "intsgd/two_kernel/bf16/int8/n8": {"bytes_per_coordinate": 38.41, "warp_instructions_per_coordinate": 5.7685},
+        "diana/fused/f32/int32/n16": {"bytes_per_coordinate": 209.244, "warp_instructions_per_coordinate": 16.073},
+        "blocks/fused/f32/int32/n16": {"bytes_per_coordinate": 75.503, "warp_instructions_per_coordinate": 9.2806},
+        "heuristic/fused/f32/int32/n16": {"bytes_per_coordinate": 139.597, "warp_instructions_per_coordinate": 9.1812},
     },
 }
 
@@ -520,39 +520,62 @@ def main():
         roofline["traffic_over_algorithmic"] = counters["bytes_per_coordinate"] * d / bytes_per_launch
         roofline["thread_instructions_per_element"] = counters["warp_instructions_per_coordinate"] * 32 / n
 
-    # ---- second limit: the 32x32->64-bit multiplies of Philox4x32-10, against their rate measured alone ----
+    # ---- second limit: the 32x32->64-bit multiplies of Philox4x32-10, against their rate measured alone, and the
+    # issue model that follows from it (on B200 nothing issues while a wide multiply does: times add up) ----
     mults = wide_multiplies_per_worker_unit(args, n)
     if mults > 0 and world == 1:
-        blocks_per_thread = 1 << 14
-        lib.intsgd_selftest_philox_rate(256, stream=stream)       # loads the kernel
-        nblocks = 0
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        t0 = time.time()
-        ev0.record()
-        for _ in range(6):
-            nblocks += lib.intsgd_selftest_philox_rate(blocks_per_thread, stream=stream)
-        ev1.record()
-        torch.cuda.synchronize()
-        t1 = time.time()
-        alone_ms = ev0.elapsed_time(ev1)
-        ck = sampler.window(t0, t1)
-        if ck["sm_mhz"]:
-            per_clock_alone = 16.0 * nblocks / (alone_ms * 1e-3 * ck["sm_mhz"] * 1e6 * sms)
+        def philox_alone(extra):
+            """Scheduler cycles one warp spends per Philox block (rounds 3-10) in the register-only kernel, with
+            `extra` independent fp32 additions per block; the SM clock is sampled while it runs."""
+            lib.intsgd_selftest_philox_rate(256, extra, stream=stream)       # loads the kernel
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            nblocks, t0 = 0, time.time()
+            ev0.record()
+            for _ in range(6):
+                nblocks += lib.intsgd_selftest_philox_rate(1 << 14, extra, stream=stream)
+            ev1.record()
+            torch.cuda.synchronize()
+            ms, ck = ev0.elapsed_time(ev1), sampler.window(t0, time.time())
+            if not ck["sm_mhz"]:
+                return None, None, ms, None
+            clocks_total = ms * 1e-3 * ck["sm_mhz"] * 1e6 * sms
+            return clocks_total * 4 / (nblocks / 32), 16.0 * nblocks / clocks_total, ms, ck["sm_mhz"]
 
+        cyc0, per_clock_alone, alone_ms, alone_mhz = philox_alone(0)
+        cyc32 = philox_alone(32)[0]
+        if cyc0 is not None:
             def per_clock(ms, mhz):
                 return mults * (n * d / 4) / (ms * 1e-3 * mhz * 1e6 * sms)
 
             co = {"bound": "alu", "unit": "32x32->64-bit products per SM clock and SM",
                   "peak": per_clock_alone, "multiplies_per_worker_unit": mults,
                   "peak_source": "rounds 3-10 of Philox4x32-10 alone (register-only kernel, 512 threads per SM, two chains "
-                                 f"per thread), {alone_ms:.0f} ms at {ck['sm_mhz']:.0f} MHz"}
+                                 f"per thread), {alone_ms:.0f} ms at {alone_mhz:.0f} MHz"}
             if clocks.get("sm_mhz"):
                 co["achieved"] = per_clock(avg_ms, clocks["sm_mhz"])
                 co["frac"] = co["achieved"] / per_clock_alone
             if sustained and sustained.get("sm_mhz_median"):
                 co["sustained_achieved"] = per_clock(sustained["ms_per_step"], sustained["sm_mhz_median"])
                 co["sustained_frac"] = co["sustained_achieved"] / per_clock_alone
+            if cyc32 is not None and counters is not None:
+                # Issue model: a warp's step time on its scheduler = Philox blocks at their measured cost + every other
+                # executed instruction at the measured cost of one more independent instruction (they do not overlap).
+                other = (cyc32 - cyc0) / 32.0
+                instr = counters["warp_instructions_per_coordinate"] * 128.0 / n      # per worker unit of a warp
+                philox_instr = 34.0 * mults / 16.0                                    # 16 multiplies + 18 logic ops per block
+                predicted = cyc0 * mults / 16.0 + (instr - philox_instr) * other
+                model = {"cycles_per_warp_philox_block": cyc0, "cycles_per_other_instruction": other,
+                         "warp_instructions_per_worker_unit": instr, "predicted_cycles_per_worker_unit": predicted,
+                         "note": "scheduler cycles per worker unit of a warp (32 units x 4 elements of one worker); "
+                                 "frac = predicted / measured"}
+                per_wuw = lambda ms, mhz: ms * 1e-3 * mhz * 1e6 * sms * 4 / (n * d / 128.0)
+                if clocks.get("sm_mhz"):
+                    model["measured_cycles_per_worker_unit"] = per_wuw(avg_ms, clocks["sm_mhz"])
+                    model["frac"] = predicted / model["measured_cycles_per_worker_unit"]
+                if sustained and sustained.get("sm_mhz_median"):
+                    model["sustained_frac"] = predicted / per_wuw(sustained["ms_per_step"], sustained["sm_mhz_median"])
+                co["issue_model"] = model
             roofline["co_limit"] = co
 
     # ---- the other rounding modes on the same buffers (context for the headline; 1 GPU only): a burst each, and the

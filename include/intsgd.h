@@ -226,9 +226,13 @@ int intsgd_selftest_wait_expiry(intsgd_ctx* ctx, void* stream);
  * when it does nothing else.  Enqueues one register-only kernel (one block of 512 threads per SM, no vector is
  * touched) in which every thread computes blocks_per_thread (2 .. 2^24, rounded down to even) blocks of rounds
  * 3-10 of Philox4x32-10 -- the per-worker part of a draw in the pipelined kernels, 16 32x32->64-bit products each --
- * as two dependent chains.  *philox_blocks (may be NULL) receives the number of blocks the launch computes; the
- * caller times the launch on `stream`.  The step kernels' random rounding cannot run faster than this rate. */
-int intsgd_selftest_philox_rate(intsgd_ctx* ctx, int64_t blocks_per_thread, int64_t* philox_blocks, void* stream);
+ * as two dependent chains.  extra_ops_per_block (0, 16 or 32) adds that many independent fp32 additions per block:
+ * the time they add tells whether other instructions hide behind the wide multiplies or queue up behind them (on
+ * B200 they queue up: one issue cycle each).  *philox_blocks (may be NULL) receives the number of blocks the launch
+ * computes; the caller times the launch on `stream`.  The step kernels' random rounding cannot run faster than the
+ * rate measured with extra_ops_per_block = 0. */
+int intsgd_selftest_philox_rate(intsgd_ctx* ctx, int64_t blocks_per_thread, int32_t extra_ops_per_block,
+                                int64_t* philox_blocks, void* stream);
 
 /* Number of kernels this library has launched on the context since creation. */
 int64_t intsgd_launch_count(const intsgd_ctx* ctx);

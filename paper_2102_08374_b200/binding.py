@@ -101,7 +101,7 @@ def load() -> C.CDLL:
     lib.intsgd_set_block_state.argtypes = [vp, vp, vp]
     lib.intsgd_sqdiff_noalloc.argtypes = [vp, vp, i64, vp, vp]
     lib.intsgd_selftest_wait_expiry.argtypes = [vp, vp]
-    lib.intsgd_selftest_philox_rate.argtypes = [vp, i64, C.POINTER(i64), vp]
+    lib.intsgd_selftest_philox_rate.argtypes = [vp, i64, i32, C.POINTER(i64), vp]
     lib.intsgd_launch_count.argtypes = [vp]
     lib.intsgd_launch_count.restype = i64
     lib.intsgd_last_error.argtypes = [vp]
@@ -349,10 +349,11 @@ class IntSGD:
     def intsgd_selftest_wait_expiry(self, stream=None):
         self._check(self._lib.intsgd_selftest_wait_expiry(self._ctx, stream))
 
-    def intsgd_selftest_philox_rate(self, blocks_per_thread, stream=None) -> int:
+    def intsgd_selftest_philox_rate(self, blocks_per_thread, extra_ops_per_block=0, stream=None) -> int:
         """Enqueue the register-only Philox kernel; returns the number of Philox blocks the launch computes."""
         count = C.c_int64(0)
-        self._check(self._lib.intsgd_selftest_philox_rate(self._ctx, blocks_per_thread, C.byref(count), stream))
+        self._check(self._lib.intsgd_selftest_philox_rate(self._ctx, blocks_per_thread, extra_ops_per_block,
+                                                          C.byref(count), stream))
         return int(count.value)
 
     def intsgd_launch_count(self) -> int:

@@ -1140,16 +1140,22 @@ int intsgd_selftest_wait_expiry(intsgd_ctx* ctx, void* stream) {
     return after_launch(ctx, "wait_expiry_kernel");
 }
 
-int intsgd_selftest_philox_rate(intsgd_ctx* ctx, int64_t blocks_per_thread, int64_t* philox_blocks, void* stream) {
+int intsgd_selftest_philox_rate(intsgd_ctx* ctx, int64_t blocks_per_thread, int32_t extra_ops_per_block,
+                                int64_t* philox_blocks, void* stream) {
     if (!ctx) return INTSGD_ERR_INVALID_ARG;
     if (blocks_per_thread < 2 || blocks_per_thread > ((int64_t)1 << 24))
         return fail(ctx, INTSGD_ERR_INVALID_ARG, "blocks_per_thread must be in 2..2^24");
+    if (extra_ops_per_block != 0 && extra_ops_per_block != 16 && extra_ops_per_block != 32)
+        return fail(ctx, INTSGD_ERR_INVALID_ARG, "extra_ops_per_block must be 0, 16 or 32");
     DeviceGuard guard(ctx->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
     ctx->last_stream = s;
     const uint32_t per_chain = (uint32_t)(blocks_per_thread / 2);
     // the sink is the state block's spare word; the kernel's store condition never holds in practice
-    philox_rate_kernel<<<ctx->sm_count, 512, 0, s>>>(ctx->keys, per_chain, &ctx->d_state->pad2);
+    uint32_t* sink = &ctx->d_state->pad2;
+    if (extra_ops_per_block == 0) philox_rate_kernel<0><<<ctx->sm_count, 512, 0, s>>>(ctx->keys, per_chain, 1e-3f, sink);
+    else if (extra_ops_per_block == 16) philox_rate_kernel<16><<<ctx->sm_count, 512, 0, s>>>(ctx->keys, per_chain, 1e-3f, sink);
+    else philox_rate_kernel<32><<<ctx->sm_count, 512, 0, s>>>(ctx->keys, per_chain, 1e-3f, sink);
     if (philox_blocks) *philox_blocks = (int64_t)ctx->sm_count * 512 * 2 * per_chain;
     return after_launch(ctx, "philox_rate_kernel");
 }

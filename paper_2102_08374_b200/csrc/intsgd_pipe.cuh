@@ -482,19 +482,30 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
 // Diagnostic: the rate at which an SM gets through rounds 3-10 of Philox4x32-10 when it does nothing else
 // (register-only: no loads, no rounding, no stores).  Every thread runs two independent chains, as a consumer of
 // the pipelined kernels does with its two units, each block's output seeding the next one's input.  The measured
-// rate of 32x32->64-bit products is the ceiling of the random-rounding kernels' arithmetic.
-__global__ void __launch_bounds__(512) philox_rate_kernel(PhiloxKeys keys, uint32_t blocks_per_chain, uint32_t* sink) {
+// rate of 32x32->64-bit products is the ceiling of the random-rounding kernels' arithmetic.  EXTRA > 0 adds that
+// many independent fp32 additions per Philox block (on eight accumulators of their own): the time they add shows
+// whether other instructions hide behind the wide multiplies or queue up behind them.
+template <int EXTRA>
+__global__ void __launch_bounds__(512) philox_rate_kernel(PhiloxKeys keys, uint32_t blocks_per_chain, float step, uint32_t* sink) {
     PhiloxThreadPart a, b;
     a.n3 = threadIdx.x; a.H = blockIdx.x; a.m1 = 0x9E3779B9u;
     b.n3 = ~threadIdx.x; b.H = blockIdx.x * 7919u; b.m1 = 0xBB67AE85u;
     uint4 ea = make_uint4(1u, 2u, 3u, 0u), eb = make_uint4(4u, 5u, 6u, 0u);
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[i] = step * (float)(i + 1) + (float)threadIdx.x;
     for (uint32_t i = 0; i < blocks_per_chain; ++i) {
         const uint4 ra = philox_finish(a, ea, keys), rb = philox_finish(b, eb, keys);
         a.H = ra.x; a.m1 = ra.y; a.n3 = ra.z; ea.z = ra.w;
         b.H = rb.x; b.m1 = rb.y; b.n3 = rb.z; eb.z = rb.w;
+#pragma unroll
+        for (int e = 0; e < 2 * EXTRA; ++e) f[e & 7] = __fadd_rn(f[e & 7], step);
     }
+    float fs = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) fs += f[i];
     // keeps the chains alive; the condition is all but impossible, so nothing is written in practice
-    if ((a.H ^ b.H ^ a.n3 ^ b.n3) == 0x5EEDu && (a.m1 ^ b.m1 ^ ea.z ^ eb.z) == 0xFACEu) *sink = a.H;
+    if ((a.H ^ b.H ^ a.n3 ^ b.n3) == 0x5EEDu && (a.m1 ^ b.m1 ^ ea.z ^ eb.z) == 0xFACEu && fs == 12345.0f) *sink = a.H;
 }
 
 // Diagnostic: the bounded wait on a barrier that nothing completes.  One thread polls `polls` times, then

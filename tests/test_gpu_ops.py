@@ -218,3 +218,20 @@ def test_an_expired_wait_is_reported_and_the_context_stays_usable():
         x_b, agg_b, st_b = two_steps(fresh)
     assert np.array_equal(x_a.view(np.uint32), x_b.view(np.uint32)) and np.array_equal(agg_a, agg_b)
     assert st_a["alpha"] == st_b["alpha"] and st_a["dx2"] == st_b["dx2"] and st_a["step"] == st_b["step"] == 2
+
+
+def test_philox_rate_diagnostic_runs_and_checks_its_arguments():
+    """The register-only Philox kernel behind the benchmark's arithmetic ceiling: it reports how many blocks a launch
+    computes, touches no vector and no state, and refuses arguments outside its documented set."""
+    with pkg.IntSGD(2, 64) as lib:
+        before = lib.intsgd_get_stats()
+        sms = torch.cuda.get_device_properties(dev()).multi_processor_count
+        for extra in (0, 16, 32):
+            assert lib.intsgd_selftest_philox_rate(64, extra) == sms * 512 * 64
+        assert lib.intsgd_selftest_philox_rate(7) == sms * 512 * 6          # rounded down to even
+        for bad in (dict(blocks_per_thread=1), dict(blocks_per_thread=(1 << 24) + 2), dict(blocks_per_thread=64, extra_ops_per_block=5)):
+            with pytest.raises(pkg.IntSGDError) as e:
+                lib.intsgd_selftest_philox_rate(**bad)
+            assert e.value.code == pkg.ERR_INVALID_ARG
+        after = lib.intsgd_get_stats()
+        assert {k: before[k] for k in ("r", "dx2", "alpha", "c", "step")} == {k: after[k] for k in ("r", "dx2", "alpha", "c", "step")}
