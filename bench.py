@@ -38,21 +38,21 @@ HBM_FALLBACK_GBS = 6650.0
 # to d, so a launch at another d is the per-coordinate figure times d.  Valid for the kernel sources with this hash:
 # any change to them makes `roofline.traffic` null until the counters are taken again.
 NCU_COUNTERS = {
-    "sources_sha256": "f7138ccd759701a69cd46cff8b9acfeedf0ea0795dd26f55554882b8a1fbb780",
+    "sources_sha256": "6b815c37c800d1efc3a2d0b090812e2b30aafeda1886355f944b9f040bdb2dee",
     "captured_log2d": 24,
     # key: kind/mode/grad/payload/n -> bytes per coordinate, warp instructions per coordinate (the vector kernels of a
     # step: fused; encode + aggregate; IntDIANA; block-wise (62 blocks); profiling pass + fused (16 bits))
     "shapes": {
-        "intsgd/fused/f32/int32/n16": {"bytes_per_coordinate": 75.39, "warp_instructions_per_coordinate": 8.1141},
-        "intsgd/fused/f32/int32/n8": {"bytes_per_coordinate": 42.9, "warp_instructions_per_coordinate": 4.3565},
-        "intsgd/fused/f32/int32/n2": {"bytes_per_coordinate": 16.997, "warp_instructions_per_coordinate": 2.0197},
-        "intsgd/fused/bf16/int8/n8": {"bytes_per_coordinate": 25.991, "warp_instructions_per_coordinate": 4.4747},
-        "intsgd/two_kernel/f32/int32/n16": {"bytes_per_coordinate": 197.937, "warp_instructions_per_coordinate": 9.8853},
-        "intsgd/two_kernel/f32/int8/n16": {"bytes_per_coordinate": 103.639, "warp_instructions_per_coordinate": 10.754},
-        "intsgd/two_kernel/bf16/int8/n8": {"bytes_per_coordinate": 38.41, "warp_instructions_per_coordinate": 5.7685},
-        "diana/fused/f32/int32/n16": {"bytes_per_coordinate": 209.244, "warp_instructions_per_coordinate": 16.073},
-        "blocks/fused/f32/int32/n16": {"bytes_per_coordinate": 75.503, "warp_instructions_per_coordinate": 9.2806},
-        "heuristic/fused/f32/int32/n16": {"bytes_per_coordinate": 139.597, "warp_instructions_per_coordinate": 9.1812},
+        "intsgd/fused/f32/int32/n16": {"bytes_per_coordinate": 75.411, "warp_instructions_per_coordinate": 8.1028},
+        "intsgd/fused/f32/int32/n8": {"bytes_per_coordinate": 42.901, "warp_instructions_per_coordinate": 4.3431},
+        "intsgd/fused/f32/int32/n2": {"bytes_per_coordinate": 16.985, "warp_instructions_per_coordinate": 2.0074},
+        "intsgd/fused/bf16/int8/n8": {"bytes_per_coordinate": 25.925, "warp_instructions_per_coordinate": 4.4393},
+        "intsgd/two_kernel/f32/int32/n16": {"bytes_per_coordinate": 197.976, "warp_instructions_per_coordinate": 9.8018},
+        "intsgd/two_kernel/f32/int8/n16": {"bytes_per_coordinate": 103.567, "warp_instructions_per_coordinate": 10.7396},
+        "intsgd/two_kernel/bf16/int8/n8": {"bytes_per_coordinate": 38.545, "warp_instructions_per_coordinate": 5.7434},
+        "diana/fused/f32/int32/n16": {"bytes_per_coordinate": 209.329, "warp_instructions_per_coordinate": 15.8897},
+        "blocks/fused/f32/int32/n16": {"bytes_per_coordinate": 75.49, "warp_instructions_per_coordinate": 9.2365},
+        "heuristic/fused/f32/int32/n16": {"bytes_per_coordinate": 139.595, "warp_instructions_per_coordinate": 9.1699},
     },
 }
 

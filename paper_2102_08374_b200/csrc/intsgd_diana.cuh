@@ -194,6 +194,7 @@ __global__ void __launch_bounds__(NC + 32, 1) diana_pipe_kernel(const __grid_con
         const uint32_t step = st->step;
         cnt_t* nonf_slot = &s_cnt[INTSGD_MAX_WORKERS];
         uint32_t s = 0, phase = 0;
+        const uint32_t full0 = smem_addr(&full_bar[0]), empty0 = smem_addr(&empty_bar[0]);
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             const int64_t unit0 = tile * kTileUnits + c;
             float4 xo[UPT], ho[UPT];
@@ -218,7 +219,7 @@ __global__ void __launch_bounds__(NC + 32, 1) diana_pipe_kernel(const __grid_con
                 S[k] = make_int4(0, 0, 0, 0);
             }
             for (int g0 = 0; g0 < n; g0 += G) {
-                if (!mbar_wait(&full_bar[s], phase)) { ok = false; break; }
+                if (!mbar_wait_at(full0 + 8u * s, phase)) { ok = false; break; }
                 const unsigned char* src = smem + (size_t)s * G * kSlot;
                 const int gw = (n - g0 < G) ? (n - g0) : G;
                 for (int w = 0; w < gw; ++w) {
@@ -238,7 +239,7 @@ __global__ void __launch_bounds__(NC + 32, 1) diana_pipe_kernel(const __grid_con
                         store_f4<true>(h_out, unit0 + (int64_t)k * NC, hn);
                     }
                 }
-                mbar_arrive(&empty_bar[s]);
+                mbar_arrive_at(empty0 + 8u * s);
                 if (++s == NS) { s = 0; phase ^= 1u; }
             }
             if (!ok) break;

@@ -93,6 +93,7 @@ __global__ void __launch_bounds__(NC + 32, 1) encode_pipe_kernel(const __grid_co
         const uint32_t step = st->step;
         const BlockParams& bp = P.bp;
         uint32_t s = 0, phase = 0;
+        const uint32_t full0 = smem_addr(&full_bar[0]), empty0 = smem_addr(&empty_bar[0]);
         for (int64_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
             const int64_t unit0 = tile * kTileUnits + c;
             PhiloxThreadPart tp[UPT];
@@ -120,7 +121,7 @@ __global__ void __launch_bounds__(NC + 32, 1) encode_pipe_kernel(const __grid_co
                 }
             }
             for (int g0 = 0; g0 < n; g0 += G) {
-                if (!mbar_wait(&full_bar[s], phase)) { ok = false; break; }
+                if (!mbar_wait_at(full0 + 8u * s, phase)) { ok = false; break; }
                 const unsigned char* src = smem + (size_t)s * G * kTileBytes;
                 const int gw = (n - g0 < G) ? (n - g0) : G;
                 // One worker's unit on the fast path: scale, round, store -- no branch, so that the G * UPT independent
@@ -166,7 +167,7 @@ __global__ void __launch_bounds__(NC + 32, 1) encode_pipe_kernel(const __grid_co
                                                            make_float4(a01[k].x, a01[k].y, a23[k].x, a23[k].y), step, s_cnt);
                     }
                 }
-                mbar_arrive(&empty_bar[s]);
+                mbar_arrive_at(empty0 + 8u * s);
                 if (++s == NS) { s = 0; phase ^= 1u; }
             }
         }

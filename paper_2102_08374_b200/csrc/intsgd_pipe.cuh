@@ -32,24 +32,35 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+// One poll.  The suspend-time hint lets the hardware park the warp for up to that long before the poll returns
+// (it returns at once when the phase completes): a waiting warp that polled in a tight loop would take issue
+// slots from the warps of its scheduler that still have work, and these kernels are bound by instruction issue.
+constexpr uint32_t kPollHintNs = 10000;
+__device__ __forceinline__ bool mbar_try_wait_at(uint32_t bar_addr, uint32_t parity) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done)
-        : "r"(smem_addr(bar)), "r"(parity)
+        : "r"(bar_addr), "r"(parity), "r"(kPollHintNs)
         : "memory");
     return done != 0;
 }
-// Bounded wait: gives up after kWaitLimit polls (each poll may itself block for a
-// hardware-defined interval), so a lost completion can never hang the GPU.
-constexpr uint32_t kWaitLimit = 1u << 22;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) { return mbar_try_wait_at(smem_addr(bar), parity); }
+// Bounded wait: gives up after kWaitLimit polls (each poll may itself block for up to the hinted interval, so
+// the bound is about ten seconds at most), so a lost completion can never hang the GPU.
+constexpr uint32_t kWaitLimit = 1u << 20;
+__device__ __forceinline__ bool mbar_wait_at(uint32_t bar_addr, uint32_t parity) {
     for (uint32_t i = 0; i < kWaitLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_at(bar_addr, parity)) return true;
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) { return mbar_wait_at(smem_addr(bar), parity); }
+// The consumers' per-stage calls take the barriers' shared-space addresses, computed once per kernel: converting
+// the generic pointer on every call costs instructions, and every instruction of these kernels costs time.
+__device__ __forceinline__ void mbar_arrive_at(uint32_t bar_addr) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_addr) : "memory");
 }
 // Programmatic dependent launch: blocks until the grids this launch depends on have completed and their
 // writes are visible; returns at once for an ordinary launch.
@@ -243,6 +254,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
         const uint32_t step = st->step;
         const BlockParams& bp = P.bp;
         uint32_t s = 0, phase = 0;
+        const uint32_t full0 = smem_addr(&full_bar[0]), empty0 = smem_addr(&empty_bar[0]);
         float max_sum = 0.0f;                                            // max |S| over fast-path units
         const bool count_overflow = P.agg_limit != 0x7FFFFFFF;          // int8 wire: count |S| > 127
         // Block-wise scales: the table entry of each of the thread's chunks and the scale of its first
@@ -307,7 +319,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                 }
             }
             for (int g0 = 0; g0 < n; g0 += G) {
-                bool arrived = mbar_wait(&full_bar[s], phase);
+                bool arrived = mbar_wait_at(full0 + 8u * s, phase);
                 if (BLOCKS) arrived = __all_sync(0xFFFFFFFFu, arrived);   // keep the warp together for the shuffles below
                 if (!arrived) { ok = false; break; }
                 const unsigned char* src = smem + (size_t)s * G * kTileBytes;
@@ -338,7 +350,7 @@ __global__ void __launch_bounds__(NC + 32, 1) fused_pipe_kernel(const __grid_con
                         }
                     }
                 }
-                mbar_arrive(&empty_bar[s]);
+                mbar_arrive_at(empty0 + 8u * s);
                 if (++s == NS) { s = 0; phase ^= 1u; }
             }
             if (!ok) break;
