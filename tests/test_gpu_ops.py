@@ -211,6 +211,14 @@ def test_an_expired_wait_is_reported_and_the_context_stays_usable():
             with pytest.raises(pkg.IntSGDError) as err:
                 lib.intsgd_get_stats()
             assert err.value.code == pkg.ERR_TIMEOUT
+        # the state block was read although the call reports the expiry: intsgd_get_state fills its output
+        import ctypes
+        from paper_2102_08374_b200 import binding
+        lib.intsgd_set_state(r=0.25, dx2=0.5, alpha=3.0, c=0.125, step=7)      # clears the flag ...
+        lib.intsgd_selftest_wait_expiry()                                       # ... and this sets it again
+        raw = binding.State(r=-1.0, dx2=-1.0, alpha=-1.0, c=-1.0, step=99, status=55)
+        assert lib._lib.intsgd_get_state(lib._ctx, ctypes.byref(raw)) == pkg.ERR_TIMEOUT
+        assert (raw.r, raw.dx2, raw.alpha, raw.c, raw.step, raw.status) == (0.25, 0.5, 3.0, 0.125, 7, pkg.OK)
         lib.intsgd_set_state(r=0.0, dx2=0.0, alpha=0.0, c=0.0, step=0)
         assert lib.intsgd_get_stats()["step"] == 0
         x_a, agg_a, st_a = two_steps(lib)
@@ -235,3 +243,21 @@ def test_philox_rate_diagnostic_runs_and_checks_its_arguments():
             assert e.value.code == pkg.ERR_INVALID_ARG
         after = lib.intsgd_get_stats()
         assert {k: before[k] for k in ("r", "dx2", "alpha", "c", "step")} == {k: after[k] for k in ("r", "dx2", "alpha", "c", "step")}
+
+
+def test_a_failed_staging_allocation_of_the_host_step_leaks_nothing():
+    """intsgd_step_host allocates its device staging on first use, all or nothing: when the buffers cannot be had
+    (here 2 x 512 GiB, more than the GPU holds) the call fails with INTSGD_ERR_CUDA before it reads a single host
+    byte, what the attempt had obtained is released, and a second attempt behaves the same."""
+    import ctypes
+    n, d = 2, 1 << 37
+    with pkg.IntSGD(n, d) as lib:
+        host = np.zeros(16, dtype=np.float32)                     # never read: the allocation fails first
+        ptrs = (ctypes.c_void_p * n)(*[host.ctypes.data] * n)
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        for _ in range(2):
+            rc = lib._lib.intsgd_step_host(lib._ctx, ptrs, host.ctypes.data, None, 0.1, pkg.MODE_EXACT, None)
+            assert rc == pkg.ERR_CUDA and "staging" in lib.intsgd_last_error()
+            free1, _ = torch.cuda.mem_get_info()
+            assert abs(free1 - free0) < (64 << 20)                # nothing of the failed attempt is kept
