@@ -366,7 +366,8 @@ def run_reference(args):
 def workload_config(args):
     kind = {"intsgd": "", "diana": ", IntDIANA step", "heuristic": f", heuristic scale with {args.num_bits} bits",
             "blocks": f", block-wise scales over {args.num_blocks} blocks"}[args.kind]
-    return {"workload": f"large-model bucket: d=2^{args.log2d} {args.grad} N(0,1e-3^2), n={args.workers} workers, "
+    row = " (the largest row of the bucket sweep)" if (args.log2d, args.workers) == (28, 16) else ""
+    return {"workload": f"large-model bucket sweep{row}: d=2^{args.log2d} {args.grad} N(0,1e-3^2), n={args.workers} workers, "
                         f"{args.payload} wire, {args.mode} path, {args.rounding} rounding{kind}",
             "d": 1 << args.log2d, "n_workers": args.workers, "grad_dtype": args.grad, "payload": args.payload,
             "mode": args.mode, "rounding": args.rounding,
